@@ -1,0 +1,120 @@
+"""The workload configurations (shapes and parameters only, no arithmetic).
+
+Five workloads mirror the benchmark definition of this repository:
+
+  tiny        2-layer fp32 ViT, 8 frames of 112x112, merge after layer 1, per-frame top-k 50 %
+  so400m_8f   SigLIP-so400m shapes, bf16, 8 frames, 30 % patch resampling
+  so400m_32f  same encoder, 32 frames (LLaVA-OneVision's frame count), 20 % resampling + brightness jitter
+  so400m_64f_p{10,50,90}  64 frames at three levels of temporal redundancy
+  serve_8x32  eight independent 32-frame videos encoded in one call, 25 % total retention
+
+The "main setting" is the hyper-parameter row of the paper's appendix table for
+25 % retention (EMA factor 0.9, segmentation threshold 0.8, merge layers
+[6, 14, 20]); the merge threshold, which the paper never prints, is a free
+parameter of the library and defaults to the segmentation threshold.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field, replace
+from typing import List, Tuple
+
+import numpy as np
+
+
+@dataclass(frozen=True)
+class EncoderShape:
+    image_size: int
+    patch_size: int
+    num_layers: int
+    hidden: int
+    heads: int
+    mlp_dim: int
+    ln_eps: float = 1e-6
+    gelu_tanh: int = 1
+    post_layernorm: int = 1
+
+    @property
+    def grid(self) -> int:
+        return self.image_size // self.patch_size
+
+    @property
+    def tokens_per_frame(self) -> int:
+        return self.grid * self.grid
+
+    @property
+    def head_dim(self) -> int:
+        return self.hidden // self.heads
+
+    @property
+    def patch_dim(self) -> int:
+        return 3 * self.patch_size * self.patch_size
+
+
+@dataclass(frozen=True)
+class MergeParams:
+    merge_layers: Tuple[int, ...] = (6, 14, 20)
+    ema_alpha: float = 0.9
+    tau_seg: float = 0.8
+    tau_merge: float = 0.8
+    weighted_merge: int = 1
+    selection: int = 1      # 0 none, 1 decoupled, 2 plain per-frame top-k
+    retain_mode: int = 1    # 0 per-frame fraction, 1 total budget
+    retain: float = 0.25
+
+
+@dataclass(frozen=True)
+class VideoSpec:
+    n_frames: int
+    resample_p: float
+    seed: int
+    jitter: float = 0.0
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    shape: EncoderShape
+    dtype: str                      # "f32" or "bf16": the arithmetic type of the CUDA path
+    videos: Tuple[VideoSpec, ...]
+    params: MergeParams
+    weight_seed: int
+    pos_std: float = 0.5
+
+    @property
+    def total_frames(self) -> int:
+        return sum(v.n_frames for v in self.videos)
+
+    def uncompressed(self) -> "Workload":
+        p = replace(self.params, merge_layers=(), selection=0, retain=1.0)
+        return replace(self, name=self.name + "_uncompressed", params=p)
+
+
+TINY = EncoderShape(image_size=112, patch_size=14, num_layers=2, hidden=64, heads=4, mlp_dim=256)
+SO400M = EncoderShape(image_size=384, patch_size=14, num_layers=27, hidden=1152, heads=16, mlp_dim=4304)
+
+MAIN = MergeParams()
+
+
+def _serve_videos() -> Tuple[VideoSpec, ...]:
+    out = []
+    for s in range(8):
+        p = float(np.random.Generator(np.random.Philox(key=1000 + s)).uniform(0.1, 0.6))
+        out.append(VideoSpec(32, round(p, 4), s))
+    return tuple(out)
+
+
+WORKLOADS = {
+    "tiny": Workload(
+        "tiny", TINY, "f32", (VideoSpec(8, 0.3, 0),),
+        MergeParams(merge_layers=(1,), selection=1, retain_mode=0, retain=0.5), 1234 + 1),
+    "so400m_8f": Workload("so400m_8f", SO400M, "bf16", (VideoSpec(8, 0.3, 0),), MAIN, 1234 + 2),
+    "so400m_32f": Workload("so400m_32f", SO400M, "bf16", (VideoSpec(32, 0.2, 0, jitter=0.05),), MAIN, 1234 + 2),
+    "so400m_64f_p10": Workload("so400m_64f_p10", SO400M, "bf16", (VideoSpec(64, 0.1, 0),), MAIN, 1234 + 2),
+    "so400m_64f_p50": Workload("so400m_64f_p50", SO400M, "bf16", (VideoSpec(64, 0.5, 0),), MAIN, 1234 + 2),
+    "so400m_64f_p90": Workload("so400m_64f_p90", SO400M, "bf16", (VideoSpec(64, 0.9, 0),), MAIN, 1234 + 2),
+    "serve_8x32": Workload("serve_8x32", SO400M, "bf16", _serve_videos(), MAIN, 1234 + 2),
+}
+
+
+def workload(name: str) -> Workload:
+    return WORKLOADS[name]
