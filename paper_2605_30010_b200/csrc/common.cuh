@@ -1,0 +1,143 @@
+// Internal declarations shared by the translation units of libearlytom (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "earlytom.h"
+
+namespace et {
+
+typedef __nv_bfloat16 bf16;
+
+extern std::atomic<unsigned long long> g_kernel_launches;
+#define ET_COUNT_LAUNCH() (::et::g_kernel_launches.fetch_add(1, std::memory_order_relaxed))
+
+// Codes written by kernels into the device status word (0 = fine).
+enum DeviceStatus : int {
+  DS_OK = 0,
+  DS_WAIT_EXPIRED = 1,      // a bounded mbarrier wait ran out
+  DS_FORCED_MISMATCH = 2,   // forced plan does not fit the frame list on the device
+  DS_CAPACITY = 3
+};
+
+static inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// Device-resident description of the current frame list (all videos of the call, concatenated).
+struct FrameList {
+  int* n;                // [1]  frames alive
+  int* vid_off;          // [Vmax+1] first frame of each video in the list
+  int* src_lo;           // [Fmax] first original frame merged into this frame (index inside its video)
+  int* src_hi;           // [Fmax]
+  unsigned char* role;   // [Fmax] 0 head, 1 middle, 2 tail, 3 single-frame segment
+};
+
+// The merge plan of one layer: how to build the next list from the current one.
+struct MergePlan {
+  int* src_a;    // [Fmax]
+  int* src_b;    // [Fmax]  -1 = copy
+  float* w_a;    // [Fmax]
+  float* w_b;    // [Fmax]
+};
+
+// Trace slot of one merge layer (device arrays [Fmax]).
+struct LayerTrace {
+  float* sim;
+  float* ema;
+  unsigned char* seg_start;
+  unsigned char* merge_next;
+};
+
+enum Epilogue : int { EPI_STORE = 0, EPI_GELU = 1, EPI_RESIDUAL = 2, EPI_TABLE = 3 };
+
+// ---- elementwise.cu ------------------------------------------------------------------------
+// frames fp32 [T][3][H][W] -> patches [T*L][k_pad] (zero padded beyond 3*p*p), fp32 or bf16.
+void launch_im2col(const float* frames, void* patches, int T, int image, int patch, int k_pad, bool out_bf16,
+                   const int* n_frames_dev, cudaStream_t s);
+// LayerNorm of rows [rows_cap][D]; live rows = *n_frames_dev * rows_per_frame when n_frames_dev != NULL.
+void launch_layernorm(const float* x, const float* g, const float* b, float eps, void* y, int rows_cap, int D,
+                      bool out_bf16, const int* n_frames_dev, int rows_per_frame, cudaStream_t s);
+
+// ---- gemm_simt.cu --------------------------------------------------------------------------
+// c = epi(a[M][K] * w[K][N] + bias) in fp32 FFMA.  live M as above.
+void launch_gemm_f32(const float* a, const float* w, const float* bias, float* c, int M_cap, int N, int K,
+                     int epilogue, int gelu_tanh, const float* table, int table_rows, const int* n_frames_dev,
+                     int rows_per_frame, cudaStream_t s);
+
+// ---- gemm_tcgen05.cu -----------------------------------------------------------------------
+struct TmaDesc { alignas(64) unsigned char bytes[128]; };
+// Build a 2-D bf16 tensor map: rows x cols (cols contiguous), box box_rows x 64 cols, 128-byte swizzle.
+bool make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                      const char** err);
+int gemm_bf16_pick_bn(int N);
+// c = epi(a[M][K] * w[N][K]^T + bias).  Descriptors must have been built for (a: M_cap x K, box 128)
+// and (w: N x K, box = gemm_bf16_pick_bn(N)).
+cudaError_t launch_gemm_bf16(const TmaDesc& da, const TmaDesc& dw, const float* bias, void* c, int M_cap, int N, int K,
+                             int epilogue, int gelu_tanh, const float* table, int table_rows, const int* n_frames_dev,
+                             int rows_per_frame, int* status_dev, cudaStream_t s);
+
+// ---- attention_simt.cu / attention_mma.cu --------------------------------------------------
+void launch_attention_f32(const float* qkv, float* out, float* lse, int n_cap, int L, int heads, int dh,
+                          const int* n_frames_dev, cudaStream_t s);
+void launch_attention_bf16(const bf16* qkv, bf16* out, float* lse, int n_cap, int L, int heads, int dh,
+                           const int* n_frames_dev, cudaStream_t s);
+bool attention_bf16_supported(int L, int heads, int dh);
+// partial[f][h][j] = sum_q exp(s(q,j) - lse[f][h][q]);  score[f][j] = sum_h partial / (heads*L)
+void launch_attention_scores_f32(const float* qkv, const float* lse, float* partial, float* score, int n_cap, int L,
+                                 int heads, int dh, const int* n_frames_dev, cudaStream_t s);
+void launch_attention_scores_bf16(const bf16* qkv, const float* lse, float* partial, float* score, int n_cap, int L,
+                                  int heads, int dh, const int* n_frames_dev, cudaStream_t s);
+
+// ---- stage1.cu -----------------------------------------------------------------------------
+void launch_token_cosines(const float* x, float* cos_scratch, int n_cap, int L, int D, const int* n_frames_dev,
+                          cudaStream_t s);
+void launch_reduce_cosines(const float* cos_scratch, float* sim, int n_cap, int L, const int* n_frames_dev,
+                           cudaStream_t s);
+struct PlanArgs {
+  const float* sim;              // [n] similarity of frames t, t+1
+  FrameList cur, nxt;
+  MergePlan plan;
+  LayerTrace trace;              // may hold NULLs
+  const unsigned char* forced_seg_start;   // NULL = decide
+  const unsigned char* forced_merge_next;
+  int forced_n_in;
+  double alpha, tau_seg, tau_merge;
+  int weighted;
+  int allow_merge;               // 0 = segmentation only (roles), list unchanged
+  int n_videos;
+  int* n_hist_slot;              // receives the new frame count (may be NULL)
+  int* status;
+};
+void launch_merge_plan(const PlanArgs& a, cudaStream_t s);
+void launch_merge_frames(const float* x, float* y, int n_cap, int frame_elems, const int* n_out_dev,
+                         const MergePlan& plan, cudaStream_t s);
+void launch_init_frames(const FrameList& fl, const int* vid_off_src_dev, int n_videos, int n_frames, cudaStream_t s);
+
+// ---- stage2.cu -----------------------------------------------------------------------------
+struct SelectSetupArgs {
+  FrameList fl;
+  const int* orig_vid_off;   // [V+1] offsets of the input videos (for B of Eq. 5)
+  int n_videos, L, selection, retain_mode;
+  double retain;
+  unsigned char* dynamic;    // [Fmax] out
+  int* k_frame;              // [Fmax] out
+  int* w_frame;              // [Fmax] out
+  int* video_k;              // [Vmax] out
+  int* video_w;              // [Vmax] out
+};
+void launch_select_setup(const SelectSetupArgs& a, int n_cap, cudaStream_t s);
+void launch_select_tokens(const float* scores, const unsigned char* dynamic, const int* k_frame, const int* w_frame,
+                          int n_cap, int L, int selection_all, unsigned char* keep, int* count,
+                          const int* n_frames_dev, cudaStream_t s);
+void launch_count_keep(const unsigned char* keep, int n_cap, int L, int* count, const int* n_frames_dev, cudaStream_t s);
+// frame_offsets[0..n] = exclusive scan of count; totals[0] = n_frames, totals[1] = n_tokens
+void launch_scan_counts(const int* count, int* frame_offsets, int* totals, int n_cap, const int* n_frames_dev,
+                        cudaStream_t s);
+void launch_gather_tokens(const float* x, const unsigned char* keep, const int* frame_offsets, int n_cap, int L, int D,
+                          const float* ln_g, const float* ln_b, float eps, float* tokens, int* token_pos,
+                          const int* n_frames_dev, cudaStream_t s);
+
+}  // namespace et

@@ -1,0 +1,83 @@
+// Patch extraction and LayerNorm kernels (HBM/L2-bound helpers around the dense layers).
+#include "common.cuh"
+#include "rowops.cuh"
+
+namespace et {
+
+// ---------------------------------------------------------------------------------------------
+// im2col: one thread per (token, channel, dy) copies the p contiguous pixels of one patch row.
+// Patch feature index = c*p*p + dy*p + dx, i.e. the flattening of a [D][3][p][p] convolution
+// weight; columns >= 3*p*p are zero (pad so that the row pitch is a multiple of 16 bytes).
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void im2col_kernel(const float* __restrict__ frames, T* __restrict__ patches, int T_frames, int image,
+                              int patch, int grid, int k_pad, const int* __restrict__ n_frames_dev) {
+  const int n_frames = n_frames_dev ? min(*n_frames_dev, T_frames) : T_frames;
+  const int L = grid * grid;
+  const int rows_per_tok = 3 * patch + 1;  // 3*p pixel rows + one job that writes the zero pad
+  const long long total = (long long)n_frames * L * rows_per_tok;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int job = (int)(idx % rows_per_tok);
+    const long long tok = idx / rows_per_tok;
+    T* dst_row = patches + tok * k_pad;
+    if (job == 3 * patch) {
+      for (int c = 3 * patch * patch; c < k_pad; ++c) dst_row[c] = to_out<T>(0.f);
+      continue;
+    }
+    const int c = job / patch, dy = job % patch;
+    const int f = (int)(tok / L), l = (int)(tok % L);
+    const int gy = l / grid, gx = l % grid;
+    const float* src = frames + (((long long)f * 3 + c) * image + (gy * patch + dy)) * image + gx * patch;
+    T* dst = dst_row + (c * patch + dy) * patch;
+    for (int dx = 0; dx < patch; ++dx) dst[dx] = to_out<T>(__ldg(src + dx));
+  }
+}
+
+void launch_im2col(const float* frames, void* patches, int T, int image, int patch, int k_pad, bool out_bf16,
+                   const int* n_frames_dev, cudaStream_t s) {
+  const int grid = image / patch;
+  const long long total = (long long)T * grid * grid * (3 * patch + 1);
+  const int threads = 256;
+  long long want = (total + threads - 1) / threads;
+  const int blocks = (int)(want < 148LL * 32 ? want : 148LL * 32);
+  if (blocks == 0) return;
+  ET_COUNT_LAUNCH();
+  if (out_bf16)
+    im2col_kernel<bf16><<<blocks, threads, 0, s>>>(frames, (bf16*)patches, T, image, patch, grid, k_pad, n_frames_dev);
+  else
+    im2col_kernel<float><<<blocks, threads, 0, s>>>(frames, (float*)patches, T, image, patch, grid, k_pad, n_frames_dev);
+}
+
+// ---------------------------------------------------------------------------------------------
+// LayerNorm: one warp per row, row held in registers, mean then centred variance (two passes over
+// registers), fp32 statistics.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void layernorm_kernel(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b,
+                                 float eps, T* __restrict__ y, int rows_cap, int D, const int* __restrict__ n_frames_dev,
+                                 int rows_per_frame) {
+  const int rows = n_frames_dev ? min(rows_cap, *n_frames_dev * rows_per_frame) : rows_cap;
+  const int warps_per_block = blockDim.x >> 5;
+  const int lane = threadIdx.x & 31;
+  for (int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5); row < rows; row += gridDim.x * warps_per_block) {
+    float4 v[ROW_MAX_VEC];
+    load_row(x + (size_t)row * D, D, lane, v);
+    layernorm_row_inplace(v, D, lane, g, b, eps);
+    store_row<T>(y + (size_t)row * D, D, lane, v);
+  }
+}
+
+void launch_layernorm(const float* x, const float* g, const float* b, float eps, void* y, int rows_cap, int D,
+                      bool out_bf16, const int* n_frames_dev, int rows_per_frame, cudaStream_t s) {
+  if (rows_cap <= 0) return;
+  const int threads = 256, wpb = threads / 32;
+  const int blocks = min(cdiv(rows_cap, wpb), 148 * 16);
+  ET_COUNT_LAUNCH();
+  if (out_bf16)
+    layernorm_kernel<bf16><<<blocks, threads, 0, s>>>(x, g, b, eps, (bf16*)y, rows_cap, D, n_frames_dev, rows_per_frame);
+  else
+    layernorm_kernel<float><<<blocks, threads, 0, s>>>(x, g, b, eps, (float*)y, rows_cap, D, n_frames_dev, rows_per_frame);
+}
+
+}  // namespace et

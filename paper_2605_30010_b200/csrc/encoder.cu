@@ -1,0 +1,703 @@
+// C-ABI entry points and host orchestration: weights, workspace, the per-call launch sequence.
+// No kernel here does arithmetic of the method; this file only sequences the kernels of the other
+// translation units on one stream and moves the (tiny) result sizes back to the host.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "rowops.cuh"
+
+namespace et {
+std::atomic<unsigned long long> g_kernel_launches{0};
+
+void launch_score_finish(const float* partial, float* score, int n_cap, int L, int heads, const int* n_frames_dev,
+                         cudaStream_t s);
+
+namespace {
+
+// dst[n][k_pad] (bf16, zero padded for k >= K) = src[k][n] (fp32)
+__global__ void transpose_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int K, int N, int k_pad) {
+  __shared__ float tile[32][33];
+  const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int k = k0 + i, n = n0 + threadIdx.x;
+    tile[i][threadIdx.x] = (k < K && n < N) ? src[(size_t)k * N + n] : 0.f;
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int n = n0 + i, k = k0 + threadIdx.x;
+    if (n < N && k < k_pad) dst[(size_t)n * k_pad + k] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+  }
+}
+
+struct LayerOffsets { size_t ln1_g, ln1_b, wqkv, bqkv, wo, bo, ln2_g, ln2_b, w1, b1, w2, b2; };
+
+struct LayerBf16 {
+  bf16 *wqkv_t, *wo_t, *w1_t, *w2_t;
+  TmaDesc d_wqkv, d_wo, d_w1, d_w2;
+};
+
+}  // namespace
+}  // namespace et
+
+using namespace et;
+
+struct et_encoder {
+  et_config cfg{};
+  int L = 0, grid = 0, P = 0, Kp = 0, dh = 0, Fmax = 0, Vmax = 0;
+  bool bf = false;
+  int device = 0;
+  std::string last_error;
+  std::vector<void*> dev_allocs, host_allocs;
+
+  // weights
+  float* w_blob = nullptr;                     // whole fp32 blob on the device (small params always read from here)
+  size_t off_patch_w = 0, off_patch_b = 0, off_pos = 0, off_post_g = 0, off_post_b = 0;
+  std::vector<LayerOffsets> lo;
+  bf16* patch_w_t = nullptr;
+  TmaDesc d_patch_w;
+  std::vector<LayerBf16> lb;
+
+  // activations
+  float* X[2] = {nullptr, nullptr};
+  void *Pm = nullptr, *Xn = nullptr, *QKV = nullptr, *O = nullptr, *Hm = nullptr;
+  TmaDesc d_Pm, d_Xn, d_O, d_Hm;
+  float *lse = nullptr, *score_partial = nullptr, *scores = nullptr, *cosbuf = nullptr, *simbuf = nullptr;
+  float* frames_stage = nullptr;               // device staging for the *_host entry point (lazy)
+
+  // frame lists, plans, traces
+  FrameList fl[2]{};
+  MergePlan plan{};
+  LayerTrace tr[ET_MAX_MERGE_LAYERS]{};
+  unsigned char* forced_seg[ET_MAX_MERGE_LAYERS]{};
+  unsigned char* forced_mrg[ET_MAX_MERGE_LAYERS]{};
+  int* orig_vid_off = nullptr;
+  unsigned char *dynamic = nullptr, *keep = nullptr;
+  int *k_frame = nullptr, *w_frame = nullptr, *video_k = nullptr, *video_w = nullptr, *count = nullptr;
+  int *frame_offsets = nullptr, *token_pos = nullptr;
+  float* tokens = nullptr;
+  int* d_small = nullptr;   // [0] n_frames, [1] n_tokens, [2..9] n after merge layer i, [10] status
+  // pinned host
+  int* h_small = nullptr;
+  int* h_vid_off = nullptr;
+  unsigned char* h_forced = nullptr;           // [2*8*Fmax]
+  unsigned char* h_keep_stage = nullptr;       // [Fmax*L]
+  // trace (host)
+  et_trace trace{};
+  float* h_tr_f = nullptr;                     // sim/ema [2*8*Fmax]
+  unsigned char* h_tr_b = nullptr;             // flags [2*8*Fmax]
+  float* h_scores = nullptr;
+  unsigned char* h_keep = nullptr;
+  int* h_video_kw = nullptr;                   // [2*Vmax]
+};
+
+namespace {
+
+et_status fail(et_encoder* e, et_status st, const std::string& msg) {
+  if (e) e->last_error = msg;
+  return st;
+}
+
+#define ET_CUDA(e, call)                                                                        \
+  do {                                                                                          \
+    cudaError_t err__ = (call);                                                                 \
+    if (err__ != cudaSuccess)                                                                   \
+      return fail((e), err__ == cudaErrorMemoryAllocation ? ET_ERR_OOM : ET_ERR_CUDA,           \
+                  std::string(#call) + ": " + cudaGetErrorString(err__));                       \
+  } while (0)
+
+template <typename T>
+et_status dalloc(et_encoder* e, T** p, size_t count) {
+  void* q = nullptr;
+  cudaError_t err = cudaMalloc(&q, std::max<size_t>(count, 1) * sizeof(T));
+  if (err != cudaSuccess) return fail(e, ET_ERR_OOM, std::string("cudaMalloc: ") + cudaGetErrorString(err));
+  e->dev_allocs.push_back(q);
+  *p = reinterpret_cast<T*>(q);
+  return ET_OK;
+}
+template <typename T>
+et_status halloc(et_encoder* e, T** p, size_t count) {
+  void* q = nullptr;
+  cudaError_t err = cudaMallocHost(&q, std::max<size_t>(count, 1) * sizeof(T));
+  if (err != cudaSuccess) return fail(e, ET_ERR_OOM, std::string("cudaMallocHost: ") + cudaGetErrorString(err));
+  e->host_allocs.push_back(q);
+  *p = reinterpret_cast<T*>(q);
+  return ET_OK;
+}
+#define ET_TRY(x)                      \
+  do {                                 \
+    et_status st__ = (x);              \
+    if (st__ != ET_OK) return st__;    \
+  } while (0)
+
+size_t blob_floats(const et_config& c, int L, int P) {
+  const size_t D = c.hidden, M = c.mlp_dim;
+  size_t per_layer = 2 * D + D * 3 * D + 3 * D + D * D + D + 2 * D + D * M + M + M * D + D;
+  return (size_t)P * D + D + (size_t)L * D + per_layer * c.num_layers + 2 * D;
+}
+
+et_status validate_config(const et_config* c) {
+  if (!c) return ET_ERR_INVALID_ARG;
+  if (c->image_size < 1 || c->patch_size < 1 || c->image_size < c->patch_size) return ET_ERR_SHAPE;
+  if (c->num_layers < 1 || c->num_layers > 64) return ET_ERR_SHAPE;
+  if (c->hidden < 4 || c->hidden % 4 != 0 || c->hidden > ROW_MAX_D) return ET_ERR_SHAPE;
+  if (c->heads < 1 || c->hidden % c->heads != 0) return ET_ERR_SHAPE;
+  if (c->hidden / c->heads > 128) return ET_ERR_SHAPE;
+  if (c->mlp_dim < 1) return ET_ERR_SHAPE;
+  if (c->dtype != ET_F32 && c->dtype != ET_BF16) return ET_ERR_INVALID_ARG;
+  if (c->dtype == ET_BF16 && (c->hidden % 8 != 0 || c->mlp_dim % 8 != 0 || (c->hidden / c->heads) % 8 != 0)) return ET_ERR_SHAPE;
+  if (c->max_frames_total < 1 || c->max_videos < 1 || c->max_videos > 1024) return ET_ERR_INVALID_ARG;
+  const long long L = (long long)(c->image_size / c->patch_size) * (c->image_size / c->patch_size);
+  if (L > 4096 || L * c->max_frames_total > (1ll << 30)) return ET_ERR_CAPACITY;
+  if (!(c->ln_eps > 0.f)) return ET_ERR_INVALID_ARG;
+  return ET_OK;
+}
+
+et_status validate_params(const et_encoder* e, const et_params* p) {
+  if (!p) return ET_ERR_INVALID_ARG;
+  if (p->num_merge_layers < 0 || p->num_merge_layers > ET_MAX_MERGE_LAYERS) return ET_ERR_INVALID_ARG;
+  for (int i = 0; i < p->num_merge_layers; ++i) {
+    if (p->merge_layers[i] < 1 || p->merge_layers[i] > e->cfg.num_layers - 1) return ET_ERR_INVALID_ARG;
+    if (i > 0 && p->merge_layers[i] <= p->merge_layers[i - 1]) return ET_ERR_INVALID_ARG;
+  }
+  if (!(p->ema_alpha > 0.0 && p->ema_alpha <= 1.0)) return ET_ERR_INVALID_ARG;
+  if (!(p->retain > 0.0 && p->retain <= 1.0)) return ET_ERR_INVALID_ARG;
+  if (isnan(p->tau_seg) || isnan(p->tau_merge)) return ET_ERR_INVALID_ARG;
+  if (p->selection < 0 || p->selection > 2) return ET_ERR_INVALID_ARG;
+  if (p->retain_mode < 0 || p->retain_mode > 1) return ET_ERR_INVALID_ARG;
+  return ET_OK;
+}
+
+// One dense layer of the encoder on the arithmetic path the encoder was created with.
+et_status dense(et_encoder* e, const void* a, const TmaDesc& da, const float* w_f32, const TmaDesc& dw,
+                const float* bias, void* c, int M_cap, int N, int K, int epi, const float* table, int table_rows,
+                const int* n_dev, cudaStream_t s) {
+  if (e->bf) {
+    ET_CUDA(e, launch_gemm_bf16(da, dw, bias, c, M_cap, N, K, epi, e->cfg.gelu_tanh, table, table_rows, n_dev, e->L,
+                                e->d_small + 10, s));
+  } else {
+    launch_gemm_f32((const float*)a, w_f32, bias, (float*)c, M_cap, N, K, epi, e->cfg.gelu_tanh, table, table_rows,
+                    n_dev, e->L, s);
+  }
+  return ET_OK;
+}
+
+et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off_host, int V, const et_params* p,
+                      cudaStream_t s, et_result* out) {
+  if (!e || !frames_dev || !vid_off_host || !out) return fail(e, ET_ERR_INVALID_ARG, "null argument");
+  ET_TRY(validate_params(e, p) == ET_OK ? ET_OK : fail(e, ET_ERR_INVALID_ARG, "invalid et_params"));
+  if (V < 1 || V > e->Vmax) return fail(e, ET_ERR_CAPACITY, "number of videos outside [1, max_videos]");
+  if (vid_off_host[0] != 0) return fail(e, ET_ERR_INVALID_ARG, "video_offsets[0] must be 0");
+  for (int v = 0; v < V; ++v)
+    if (vid_off_host[v + 1] <= vid_off_host[v]) return fail(e, ET_ERR_INVALID_ARG, "every video needs at least one frame");
+  const int T = vid_off_host[V];
+  if (T > e->Fmax) return fail(e, ET_ERR_CAPACITY, "more frames than max_frames_total");
+  const et_forced_plan* fp = p->forced_plan;
+  if (fp) {
+    for (int i = 0; i < p->num_merge_layers; ++i) {
+      if (!fp->seg_start[i] || !fp->merge_next[i] || fp->n_in[i] < 1 || fp->n_in[i] > T)
+        return fail(e, ET_ERR_INVALID_ARG, "forced plan: missing or oversized layer entry");
+      for (int t = 0; t < fp->n_in[i]; ++t)
+        if (fp->merge_next[i][t] && (t + 1 >= fp->n_in[i] || fp->merge_next[i][t + 1]))
+          return fail(e, ET_ERR_INVALID_ARG, "forced plan: overlapping or dangling merge pair");
+    }
+    if (fp->keep && (fp->n_final < 1 || fp->n_final > T)) return fail(e, ET_ERR_INVALID_ARG, "forced plan: n_final");
+  }
+  ET_CUDA(e, cudaSetDevice(e->device));
+
+  const et_config& c = e->cfg;
+  const int L = e->L, D = c.hidden, Mlp = c.mlp_dim, H = c.heads, dh = e->dh;
+  const int rows_cap = T * L;
+  const float* W = e->w_blob;
+
+  memcpy(e->h_vid_off, vid_off_host, sizeof(int) * (V + 1));
+  ET_CUDA(e, cudaMemcpyAsync(e->orig_vid_off, e->h_vid_off, sizeof(int) * (V + 1), cudaMemcpyHostToDevice, s));
+  ET_CUDA(e, cudaMemsetAsync(e->d_small, 0, sizeof(int) * 16, s));
+  if (fp) {
+    for (int i = 0; i < p->num_merge_layers; ++i) {
+      unsigned char* hs = e->h_forced + (size_t)(2 * i) * e->Fmax;
+      unsigned char* hm = e->h_forced + (size_t)(2 * i + 1) * e->Fmax;
+      memcpy(hs, fp->seg_start[i], fp->n_in[i]);
+      memcpy(hm, fp->merge_next[i], fp->n_in[i]);
+      ET_CUDA(e, cudaMemcpyAsync(e->forced_seg[i], hs, fp->n_in[i], cudaMemcpyHostToDevice, s));
+      ET_CUDA(e, cudaMemcpyAsync(e->forced_mrg[i], hm, fp->n_in[i], cudaMemcpyHostToDevice, s));
+    }
+  }
+  int lst = 0, cur = 0;
+  launch_init_frames(e->fl[0], e->orig_vid_off, V, T, s);
+
+  // patch embedding: im2col + dense layer with the position table added in the epilogue
+  launch_im2col(frames_dev, e->Pm, T, c.image_size, c.patch_size, e->Kp, e->bf, nullptr, s);
+  ET_TRY(dense(e, e->Pm, e->d_Pm, W + e->off_patch_w, e->d_patch_w, W + e->off_patch_b, e->X[cur], rows_cap, D,
+               e->bf ? e->Kp : e->P, EPI_TABLE, W + e->off_pos, L, nullptr, s));
+
+  int mi = 0;
+  for (int layer = 0; layer < c.num_layers; ++layer) {
+    if (mi < p->num_merge_layers && p->merge_layers[mi] == layer) {
+      // Stage I at this block: similarities -> plan -> weighted merge + compaction
+      const int* n_dev = e->fl[lst].n;
+      launch_token_cosines(e->X[cur], e->cosbuf, T, L, D, n_dev, s);
+      launch_reduce_cosines(e->cosbuf, e->simbuf, T, L, n_dev, s);
+      PlanArgs a{};
+      a.sim = e->simbuf; a.cur = e->fl[lst]; a.nxt = e->fl[lst ^ 1]; a.plan = e->plan; a.trace = e->tr[mi];
+      a.forced_seg_start = fp ? e->forced_seg[mi] : nullptr;
+      a.forced_merge_next = fp ? e->forced_mrg[mi] : nullptr;
+      a.forced_n_in = fp ? fp->n_in[mi] : 0;
+      a.alpha = p->ema_alpha; a.tau_seg = p->tau_seg; a.tau_merge = p->tau_merge;
+      a.weighted = p->weighted_merge; a.allow_merge = 1; a.n_videos = V;
+      a.n_hist_slot = e->d_small + 2 + mi; a.status = e->d_small + 10;
+      launch_merge_plan(a, s);
+      launch_merge_frames(e->X[cur], e->X[cur ^ 1], T, L * D, e->fl[lst ^ 1].n, e->plan, s);
+      cur ^= 1; lst ^= 1; ++mi;
+    }
+    const int* n_dev = e->fl[lst].n;
+    const LayerOffsets& o = e->lo[layer];
+    const LayerBf16* b = e->bf ? &e->lb[layer] : nullptr;
+    static const TmaDesc none{};
+    launch_layernorm(e->X[cur], W + o.ln1_g, W + o.ln1_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s);
+    ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.wqkv, b ? b->d_wqkv : none, W + o.bqkv, e->QKV, rows_cap, 3 * D, D, EPI_STORE,
+                 nullptr, 1, n_dev, s));
+    if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, s);
+    else launch_attention_f32((const float*)e->QKV, (float*)e->O, e->lse, T, L, H, dh, n_dev, s);
+    if (layer == c.num_layers - 1) {
+      if (e->bf) launch_attention_scores_bf16((const bf16*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
+      else launch_attention_scores_f32((const float*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
+    }
+    ET_TRY(dense(e, e->O, e->d_O, W + o.wo, b ? b->d_wo : none, W + o.bo, e->X[cur], rows_cap, D, D, EPI_RESIDUAL,
+                 nullptr, 1, n_dev, s));
+    launch_layernorm(e->X[cur], W + o.ln2_g, W + o.ln2_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s);
+    ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, W + o.b1, e->Hm, rows_cap, Mlp, D, EPI_GELU, nullptr, 1,
+                 n_dev, s));
+    ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, W + o.b2, e->X[cur], rows_cap, D, Mlp, EPI_RESIDUAL,
+                 nullptr, 1, n_dev, s));
+  }
+  const int* n_dev = e->fl[lst].n;
+  if (p->num_merge_layers == 0) {
+    // Stage I off: the segment list of Stage II comes from the streaming segmentation of the final features
+    launch_token_cosines(e->X[cur], e->cosbuf, T, L, D, n_dev, s);
+    launch_reduce_cosines(e->cosbuf, e->simbuf, T, L, n_dev, s);
+    PlanArgs a{};
+    a.sim = e->simbuf; a.cur = e->fl[lst]; a.nxt = e->fl[lst ^ 1]; a.plan = e->plan; a.trace = e->tr[0];
+    a.alpha = p->ema_alpha; a.tau_seg = p->tau_seg; a.tau_merge = p->tau_merge;
+    a.weighted = p->weighted_merge; a.allow_merge = 0; a.n_videos = V; a.status = e->d_small + 10;
+    launch_merge_plan(a, s);
+  }
+  // Stage II
+  SelectSetupArgs sa{};
+  sa.fl = e->fl[lst]; sa.orig_vid_off = e->orig_vid_off; sa.n_videos = V; sa.L = L; sa.selection = p->selection;
+  sa.retain_mode = p->retain_mode; sa.retain = p->retain; sa.dynamic = e->dynamic; sa.k_frame = e->k_frame;
+  sa.w_frame = e->w_frame; sa.video_k = e->video_k; sa.video_w = e->video_w;
+  launch_select_setup(sa, T, s);
+  if (fp && fp->keep) {
+    memcpy(e->h_keep_stage, fp->keep, (size_t)fp->n_final * L);
+    ET_CUDA(e, cudaMemcpyAsync(e->keep, e->h_keep_stage, (size_t)fp->n_final * L, cudaMemcpyHostToDevice, s));
+    launch_count_keep(e->keep, T, L, e->count, n_dev, s);
+  } else {
+    if (p->selection == 2) ET_CUDA(e, cudaMemsetAsync(e->dynamic, 1, T, s));   // plain top-k: every frame ranks globally
+    launch_select_tokens(e->scores, e->dynamic, e->k_frame, e->w_frame, T, L, p->selection == 0, e->keep, e->count, n_dev, s);
+    if (p->selection == 2) launch_select_setup(sa, T, s);                      // restore the reported dynamic flags
+  }
+  launch_scan_counts(e->count, e->frame_offsets, e->d_small, T, n_dev, s);
+  launch_gather_tokens(e->X[cur], e->keep, e->frame_offsets, T, L, D, c.post_layernorm ? W + e->off_post_g : nullptr,
+                       c.post_layernorm ? W + e->off_post_b : nullptr, c.ln_eps, e->tokens, e->token_pos, n_dev, s);
+  ET_CUDA(e, cudaMemcpyAsync(e->h_small, e->d_small, sizeof(int) * 16, cudaMemcpyDeviceToHost, s));
+  ET_CUDA(e, cudaGetLastError());
+  ET_CUDA(e, cudaStreamSynchronize(s));
+
+  const int status = e->h_small[10];
+  if (status == DS_WAIT_EXPIRED) return fail(e, ET_ERR_TIMEOUT, "a bounded device-side wait expired in a tensor-core kernel");
+  if (status == DS_FORCED_MISMATCH) return fail(e, ET_ERR_INVALID_ARG, "forced plan does not fit the frame list");
+  if (status != 0) return fail(e, ET_ERR_CUDA, "device status " + std::to_string(status));
+  const int N = e->h_small[0], n_tok = e->h_small[1];
+  if (fp && fp->keep && fp->n_final != N) return fail(e, ET_ERR_INVALID_ARG, "forced plan: n_final does not match");
+
+  et_result r{};
+  r.n_videos = V; r.n_frames_in = T; r.n_frames_out = N; r.n_tokens = n_tok; r.hidden = D; r.tokens_per_frame = L;
+  r.tokens = e->tokens; r.video_frame_offsets = e->fl[lst].vid_off; r.frame_offsets = e->frame_offsets;
+  r.frame_src_lo = e->fl[lst].src_lo; r.frame_src_hi = e->fl[lst].src_hi; r.frame_dynamic = e->dynamic;
+  r.token_pos = e->token_pos; r.trace = nullptr;
+  {
+    int alive = T, m = 0;
+    for (int layer = 0; layer < c.num_layers; ++layer) {
+      if (m < p->num_merge_layers && p->merge_layers[m] == layer) { alive = e->h_small[2 + m]; ++m; }
+      r.frames_per_block[layer] = alive;
+    }
+  }
+  if (p->want_trace) {
+    et_trace& t = e->trace;
+    memset(&t, 0, sizeof(t));
+    t.num_merge_layers = p->num_merge_layers;
+    int n_in = T;
+    for (int i = 0; i < p->num_merge_layers; ++i) {
+      t.n_in[i] = n_in; t.n_out[i] = e->h_small[2 + i];
+      float* hs = e->h_tr_f + (size_t)(2 * i) * e->Fmax;
+      float* he = e->h_tr_f + (size_t)(2 * i + 1) * e->Fmax;
+      unsigned char* hb = e->h_tr_b + (size_t)(2 * i) * e->Fmax;
+      unsigned char* hm = e->h_tr_b + (size_t)(2 * i + 1) * e->Fmax;
+      ET_CUDA(e, cudaMemcpyAsync(hs, e->tr[i].sim, sizeof(float) * n_in, cudaMemcpyDeviceToHost, s));
+      ET_CUDA(e, cudaMemcpyAsync(he, e->tr[i].ema, sizeof(float) * n_in, cudaMemcpyDeviceToHost, s));
+      ET_CUDA(e, cudaMemcpyAsync(hb, e->tr[i].seg_start, n_in, cudaMemcpyDeviceToHost, s));
+      ET_CUDA(e, cudaMemcpyAsync(hm, e->tr[i].merge_next, n_in, cudaMemcpyDeviceToHost, s));
+      t.sim[i] = hs; t.ema[i] = he; t.seg_start[i] = hb; t.merge_next[i] = hm;
+      n_in = t.n_out[i];
+    }
+    ET_CUDA(e, cudaMemcpyAsync(e->h_scores, e->scores, sizeof(float) * (size_t)N * L, cudaMemcpyDeviceToHost, s));
+    ET_CUDA(e, cudaMemcpyAsync(e->h_keep, e->keep, (size_t)N * L, cudaMemcpyDeviceToHost, s));
+    ET_CUDA(e, cudaMemcpyAsync(e->h_video_kw, e->video_k, sizeof(int) * V, cudaMemcpyDeviceToHost, s));
+    ET_CUDA(e, cudaMemcpyAsync(e->h_video_kw + e->Vmax, e->video_w, sizeof(int) * V, cudaMemcpyDeviceToHost, s));
+    ET_CUDA(e, cudaStreamSynchronize(s));
+    t.scores = e->h_scores; t.keep = e->h_keep; t.video_k = e->h_video_kw; t.video_w = e->h_video_kw + e->Vmax;
+    r.trace = &t;
+  }
+  *out = r;
+  return ET_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+et_status et_encoder_create(const et_config* config, const et_weights* weights, et_encoder** out) {
+  if (!config || !weights || !weights->data || !out) return ET_ERR_INVALID_ARG;
+  et_status st = validate_config(config);
+  if (st != ET_OK) return st;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return ET_ERR_CUDA;
+  const int g = config->image_size / config->patch_size;
+  const int L = g * g, P = 3 * config->patch_size * config->patch_size;
+  if (weights->count != blob_floats(*config, L, P)) return ET_ERR_WEIGHTS;
+
+  et_encoder* e = new (std::nothrow) et_encoder();
+  if (!e) return ET_ERR_OOM;
+  auto bail = [&](et_status s) { et_destroy(e); return s; };
+  e->cfg = *config;
+  e->L = L; e->grid = g; e->P = P; e->dh = config->hidden / config->heads;
+  e->bf = config->dtype == ET_BF16;
+  e->Kp = e->bf ? (P + 7) / 8 * 8 : P;
+  e->Fmax = config->max_frames_total; e->Vmax = config->max_videos;
+  if (cudaGetDevice(&e->device) != cudaSuccess) return bail(ET_ERR_CUDA);
+  const size_t D = config->hidden, M = config->mlp_dim, F = e->Fmax, rows = F * (size_t)L;
+
+  // ---- weights
+  {
+    size_t off = 0;
+    auto take = [&](size_t n) { size_t o = off; off += n; return o; };
+    e->off_patch_w = take((size_t)P * D); e->off_patch_b = take(D); e->off_pos = take((size_t)L * D);
+    e->lo.resize(config->num_layers);
+    for (auto& o : e->lo) {
+      o.ln1_g = take(D); o.ln1_b = take(D); o.wqkv = take(D * 3 * D); o.bqkv = take(3 * D);
+      o.wo = take(D * D); o.bo = take(D); o.ln2_g = take(D); o.ln2_b = take(D);
+      o.w1 = take(D * M); o.b1 = take(M); o.w2 = take(M * D); o.b2 = take(D);
+    }
+    e->off_post_g = take(D); e->off_post_b = take(D);
+  }
+  if ((st = dalloc(e, &e->w_blob, weights->count)) != ET_OK) return bail(st);
+  if (cudaMemcpy(e->w_blob, weights->data, weights->count * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+    return bail(ET_ERR_CUDA);
+  const size_t es = e->bf ? 2 : 4;
+  // ---- activations
+  void* tmp = nullptr;
+#define ET_A(ptr, bytes)                                                     \
+  do {                                                                       \
+    unsigned char* q__ = nullptr;                                            \
+    if ((st = dalloc(e, &q__, (bytes))) != ET_OK) return bail(st);           \
+    ptr = reinterpret_cast<decltype(ptr)>(q__);                              \
+  } while (0)
+  ET_A(e->X[0], rows * D * 4); ET_A(e->X[1], rows * D * 4);
+  ET_A(e->Pm, rows * e->Kp * es); ET_A(e->Xn, rows * D * es); ET_A(e->QKV, rows * 3 * D * es);
+  ET_A(e->O, rows * D * es); ET_A(e->Hm, rows * M * es);
+  ET_A(e->lse, F * config->heads * L * 4); ET_A(e->score_partial, F * config->heads * L * 4);
+  ET_A(e->scores, rows * 4); ET_A(e->cosbuf, rows * 4); ET_A(e->simbuf, F * 4);
+  for (int i = 0; i < 2; ++i) {
+    ET_A(e->fl[i].n, 4); ET_A(e->fl[i].vid_off, (e->Vmax + 1) * 4); ET_A(e->fl[i].src_lo, F * 4);
+    ET_A(e->fl[i].src_hi, F * 4); ET_A(e->fl[i].role, F);
+  }
+  ET_A(e->plan.src_a, F * 4); ET_A(e->plan.src_b, F * 4); ET_A(e->plan.w_a, F * 4); ET_A(e->plan.w_b, F * 4);
+  for (int i = 0; i < ET_MAX_MERGE_LAYERS; ++i) {
+    ET_A(e->tr[i].sim, F * 4); ET_A(e->tr[i].ema, F * 4); ET_A(e->tr[i].seg_start, F); ET_A(e->tr[i].merge_next, F);
+    ET_A(e->forced_seg[i], F); ET_A(e->forced_mrg[i], F);
+  }
+  ET_A(e->orig_vid_off, (e->Vmax + 1) * 4);
+  ET_A(e->dynamic, F); ET_A(e->keep, rows); ET_A(e->k_frame, F * 4); ET_A(e->w_frame, F * 4);
+  ET_A(e->video_k, e->Vmax * 4); ET_A(e->video_w, e->Vmax * 4); ET_A(e->count, F * 4);
+  ET_A(e->frame_offsets, (F + 1) * 4); ET_A(e->token_pos, rows * 4); ET_A(e->tokens, rows * D * 4);
+  ET_A(e->d_small, 16 * 4);
+#undef ET_A
+  (void)tmp;
+  if ((st = halloc(e, &e->h_small, 16)) != ET_OK) return bail(st);
+  if ((st = halloc(e, &e->h_vid_off, e->Vmax + 1)) != ET_OK) return bail(st);
+  if ((st = halloc(e, &e->h_forced, 2 * ET_MAX_MERGE_LAYERS * F)) != ET_OK) return bail(st);
+  if ((st = halloc(e, &e->h_keep_stage, rows)) != ET_OK) return bail(st);
+  if ((st = halloc(e, &e->h_tr_f, 2 * ET_MAX_MERGE_LAYERS * F)) != ET_OK) return bail(st);
+  if ((st = halloc(e, &e->h_tr_b, 2 * ET_MAX_MERGE_LAYERS * F)) != ET_OK) return bail(st);
+  if ((st = halloc(e, &e->h_scores, rows)) != ET_OK) return bail(st);
+  if ((st = halloc(e, &e->h_keep, rows)) != ET_OK) return bail(st);
+  if ((st = halloc(e, &e->h_video_kw, 2 * (size_t)e->Vmax)) != ET_OK) return bail(st);
+  // zero the activation buffers once: rows beyond the live count are read (never stored) by tile loads
+  cudaMemset(e->Pm, 0, rows * e->Kp * es); cudaMemset(e->Xn, 0, rows * D * es); cudaMemset(e->O, 0, rows * D * es);
+  cudaMemset(e->Hm, 0, rows * M * es); cudaMemset(e->QKV, 0, rows * 3 * D * es);
+
+  if (e->bf) {
+    // transposed bf16 copies of the dense weights ([out][in], K contiguous) + their tensor maps
+    const char* err = nullptr;
+    auto convert = [&](size_t off, int K, int N, int k_pad, bf16** dst) -> et_status {
+      et_status s2 = dalloc(e, dst, (size_t)N * k_pad);
+      if (s2 != ET_OK) return s2;
+      ET_COUNT_LAUNCH();
+      transpose_to_bf16_kernel<<<dim3(cdiv(N, 32), cdiv(k_pad, 32)), dim3(32, 8)>>>(e->w_blob + off, *dst, K, N, k_pad);
+      return cudaGetLastError() == cudaSuccess ? ET_OK : ET_ERR_CUDA;
+    };
+    if ((st = convert(e->off_patch_w, P, (int)D, e->Kp, &e->patch_w_t)) != ET_OK) return bail(st);
+    if (!make_tma_2d_bf16(&e->d_patch_w, e->patch_w_t, D, e->Kp, gemm_bf16_pick_bn((int)D), &err)) return bail(fail(e, ET_ERR_CUDA, err));
+    e->lb.resize(config->num_layers);
+    for (int i = 0; i < config->num_layers; ++i) {
+      LayerBf16& b = e->lb[i];
+      const LayerOffsets& o = e->lo[i];
+      if ((st = convert(o.wqkv, (int)D, (int)(3 * D), (int)D, &b.wqkv_t)) != ET_OK) return bail(st);
+      if ((st = convert(o.wo, (int)D, (int)D, (int)D, &b.wo_t)) != ET_OK) return bail(st);
+      if ((st = convert(o.w1, (int)D, (int)M, (int)D, &b.w1_t)) != ET_OK) return bail(st);
+      if ((st = convert(o.w2, (int)M, (int)D, (int)M, &b.w2_t)) != ET_OK) return bail(st);
+      bool ok = make_tma_2d_bf16(&b.d_wqkv, b.wqkv_t, 3 * D, D, gemm_bf16_pick_bn((int)(3 * D)), &err) &&
+                make_tma_2d_bf16(&b.d_wo, b.wo_t, D, D, gemm_bf16_pick_bn((int)D), &err) &&
+                make_tma_2d_bf16(&b.d_w1, b.w1_t, M, D, gemm_bf16_pick_bn((int)M), &err) &&
+                make_tma_2d_bf16(&b.d_w2, b.w2_t, D, M, gemm_bf16_pick_bn((int)D), &err);
+      if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
+    }
+    bool ok = make_tma_2d_bf16(&e->d_Pm, e->Pm, rows, e->Kp, 128, &err) && make_tma_2d_bf16(&e->d_Xn, e->Xn, rows, D, 128, &err) &&
+              make_tma_2d_bf16(&e->d_O, e->O, rows, D, 128, &err) && make_tma_2d_bf16(&e->d_Hm, e->Hm, rows, M, 128, &err);
+    if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
+  }
+  if (cudaDeviceSynchronize() != cudaSuccess) return bail(ET_ERR_CUDA);
+  *out = e;
+  return ET_OK;
+}
+
+void et_destroy(et_encoder* e) {
+  if (!e) return;
+  for (void* p : e->dev_allocs) cudaFree(p);
+  for (void* p : e->host_allocs) cudaFreeHost(p);
+  delete e;
+}
+
+et_status et_encode_batch(et_encoder* enc, const float* frames_dev, const int* video_offsets_host, int V,
+                          const et_params* params, void* cuda_stream, et_result* out) {
+  return encode_impl(enc, frames_dev, video_offsets_host, V, params, (cudaStream_t)cuda_stream, out);
+}
+
+et_status et_encode_video(et_encoder* enc, const float* frames_dev, int T, const et_params* params, void* cuda_stream,
+                          et_result* out) {
+  if (T < 1) return fail(enc, ET_ERR_INVALID_ARG, "T < 1");
+  const int offs[2] = {0, T};
+  return encode_impl(enc, frames_dev, offs, 1, params, (cudaStream_t)cuda_stream, out);
+}
+
+et_status et_encode_batch_host(et_encoder* e, const float* frames_host, const int* video_offsets_host, int V,
+                               const et_params* params, void* cuda_stream, const et_host_buffers* dst, et_result* out) {
+  if (!e || !frames_host || !video_offsets_host || !dst || !out) return fail(e, ET_ERR_INVALID_ARG, "null argument");
+  if (V < 1 || V > e->Vmax) return fail(e, ET_ERR_CAPACITY, "number of videos outside [1, max_videos]");
+  const int T = video_offsets_host[V];
+  if (T < 1 || T > e->Fmax) return fail(e, ET_ERR_CAPACITY, "frames outside [1, max_frames_total]");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const size_t frame_floats = (size_t)3 * e->cfg.image_size * e->cfg.image_size;
+  if (!e->frames_stage) ET_TRY(dalloc(e, &e->frames_stage, (size_t)e->Fmax * frame_floats));
+  ET_CUDA(e, cudaMemcpyAsync(e->frames_stage, frames_host, (size_t)T * frame_floats * sizeof(float), cudaMemcpyHostToDevice, s));
+  et_result r{};
+  ET_TRY(encode_impl(e, e->frames_stage, video_offsets_host, V, params, s, &r));
+  if ((size_t)r.n_tokens > dst->capacity_tokens || (size_t)r.n_frames_out > dst->capacity_frames)
+    return fail(e, ET_ERR_CAPACITY, "host buffers too small for the result");
+  const size_t N = r.n_frames_out, nt = r.n_tokens;
+  if (dst->tokens) ET_CUDA(e, cudaMemcpyAsync(dst->tokens, r.tokens, nt * r.hidden * sizeof(float), cudaMemcpyDeviceToHost, s));
+  if (dst->token_pos) ET_CUDA(e, cudaMemcpyAsync(dst->token_pos, r.token_pos, nt * sizeof(int), cudaMemcpyDeviceToHost, s));
+  if (dst->frame_offsets) ET_CUDA(e, cudaMemcpyAsync(dst->frame_offsets, r.frame_offsets, (N + 1) * sizeof(int), cudaMemcpyDeviceToHost, s));
+  if (dst->frame_src_lo) ET_CUDA(e, cudaMemcpyAsync(dst->frame_src_lo, r.frame_src_lo, N * sizeof(int), cudaMemcpyDeviceToHost, s));
+  if (dst->frame_src_hi) ET_CUDA(e, cudaMemcpyAsync(dst->frame_src_hi, r.frame_src_hi, N * sizeof(int), cudaMemcpyDeviceToHost, s));
+  if (dst->frame_dynamic) ET_CUDA(e, cudaMemcpyAsync(dst->frame_dynamic, r.frame_dynamic, N, cudaMemcpyDeviceToHost, s));
+  if (dst->video_frame_offsets)
+    ET_CUDA(e, cudaMemcpyAsync(dst->video_frame_offsets, r.video_frame_offsets, (V + 1) * sizeof(int), cudaMemcpyDeviceToHost, s));
+  ET_CUDA(e, cudaStreamSynchronize(s));
+  *out = r;
+  return ET_OK;
+}
+
+const char* et_status_string(et_status s) {
+  switch (s) {
+    case ET_OK: return "ok";
+    case ET_ERR_INVALID_ARG: return "invalid argument";
+    case ET_ERR_SHAPE: return "inconsistent shape";
+    case ET_ERR_CAPACITY: return "capacity exceeded";
+    case ET_ERR_OOM: return "out of memory";
+    case ET_ERR_CUDA: return "CUDA error";
+    case ET_ERR_TIMEOUT: return "device-side wait expired";
+    case ET_ERR_WEIGHTS: return "bad weight blob";
+  }
+  return "unknown status";
+}
+
+const char* et_last_error(const et_encoder* enc) { return enc ? enc->last_error.c_str() : ""; }
+
+unsigned long long et_kernel_launch_count(void) { return g_kernel_launches.load(); }
+
+// ------------------------------------------------------------------------------------------------
+// single steps
+// ------------------------------------------------------------------------------------------------
+#define ET_CUDA0(call)                                 \
+  do {                                                 \
+    if ((call) != cudaSuccess) return ET_ERR_CUDA;     \
+  } while (0)
+
+et_status et_frame_similarity(const float* x_dev, int n, int L, int D, float* cos_scratch_dev, float* sim_dev,
+                              void* cuda_stream) {
+  if (!x_dev || !cos_scratch_dev || !sim_dev) return ET_ERR_INVALID_ARG;
+  if (n < 1 || L < 1 || D < 4 || D % 4 != 0 || D > ROW_MAX_D) return ET_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  launch_token_cosines(x_dev, cos_scratch_dev, n, L, D, nullptr, s);
+  launch_reduce_cosines(cos_scratch_dev, sim_dev, n, L, nullptr, s);
+  ET_CUDA0(cudaGetLastError());
+  return ET_OK;
+}
+
+et_status et_merge_plan(const float* sim_dev, const int* video_offsets_dev, int n, int V, double ema_alpha, double tau_seg,
+                        double tau_merge, int weighted_merge, unsigned char* seg_start_dev, unsigned char* merge_next_dev,
+                        float* ema_dev, int* n_out_dev, int* src_a_dev, int* src_b_dev, float* w_a_dev, float* w_b_dev,
+                        int* new_video_offsets_dev, void* cuda_stream) {
+  if (!sim_dev || !video_offsets_dev || !seg_start_dev || !merge_next_dev || !ema_dev || !n_out_dev || !src_a_dev ||
+      !src_b_dev || !w_a_dev || !w_b_dev || !new_video_offsets_dev)
+    return ET_ERR_INVALID_ARG;
+  if (n < 1 || V < 1 || V > 1024) return ET_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  // scratch for the list bookkeeping this entry point does not expose
+  int* scratch = nullptr;
+  const size_t ints = 2 + 4 * (size_t)n + (size_t)n /*sim copy as float*/ + 2;
+  ET_CUDA0(cudaMalloc(&scratch, ints * sizeof(int) + 2 * (size_t)n));
+  int* n_cur = scratch;
+  int* status = scratch + 1;
+  int* lo0 = scratch + 2; int* hi0 = lo0 + n; int* lo1 = hi0 + n; int* hi1 = lo1 + n;
+  float* sim_tr = reinterpret_cast<float*>(hi1 + n);
+  unsigned char* role0 = reinterpret_cast<unsigned char*>(sim_tr + n + 2);
+  unsigned char* role1 = role0 + n;
+  cudaMemsetAsync(scratch, 0, ints * sizeof(int) + 2 * (size_t)n, s);
+  cudaMemcpyAsync(n_cur, &n, sizeof(int), cudaMemcpyHostToDevice, s);
+  PlanArgs a{};
+  a.sim = sim_dev;
+  a.cur = FrameList{n_cur, const_cast<int*>(video_offsets_dev), lo0, hi0, role0};
+  a.nxt = FrameList{n_out_dev, new_video_offsets_dev, lo1, hi1, role1};
+  a.plan = MergePlan{src_a_dev, src_b_dev, w_a_dev, w_b_dev};
+  a.trace = LayerTrace{sim_tr, ema_dev, seg_start_dev, merge_next_dev};
+  a.alpha = ema_alpha; a.tau_seg = tau_seg; a.tau_merge = tau_merge; a.weighted = weighted_merge;
+  a.allow_merge = 1; a.n_videos = V; a.status = status;
+  launch_merge_plan(a, s);
+  cudaError_t err = cudaStreamSynchronize(s);
+  cudaFree(scratch);
+  return err == cudaSuccess ? ET_OK : ET_ERR_CUDA;
+}
+
+et_status et_merge_frames(const float* x_dev, float* y_dev, int n_cap, int frame_elems, const int* n_out_dev,
+                          const int* src_a_dev, const int* src_b_dev, const float* w_a_dev, const float* w_b_dev,
+                          void* cuda_stream) {
+  if (!x_dev || !y_dev || !n_out_dev || !src_a_dev || !src_b_dev || !w_a_dev || !w_b_dev || x_dev == y_dev) return ET_ERR_INVALID_ARG;
+  if (n_cap < 1 || n_cap > 65535 || frame_elems < 4 || frame_elems % 4 != 0) return ET_ERR_SHAPE;
+  MergePlan p{const_cast<int*>(src_a_dev), const_cast<int*>(src_b_dev), const_cast<float*>(w_a_dev), const_cast<float*>(w_b_dev)};
+  launch_merge_frames(x_dev, y_dev, n_cap, frame_elems, n_out_dev, p, (cudaStream_t)cuda_stream);
+  ET_CUDA0(cudaGetLastError());
+  return ET_OK;
+}
+
+et_status et_select_tokens(const float* scores_dev, const unsigned char* dynamic_dev, const int* k_dev, const int* w_dev,
+                           int N, int L, unsigned char* keep_dev, int* count_dev, void* cuda_stream) {
+  if (!scores_dev || !dynamic_dev || !k_dev || !w_dev || !keep_dev || !count_dev) return ET_ERR_INVALID_ARG;
+  if (N < 1 || L < 1 || L > 4096) return ET_ERR_SHAPE;
+  launch_select_tokens(scores_dev, dynamic_dev, k_dev, w_dev, N, L, 0, keep_dev, count_dev, nullptr, (cudaStream_t)cuda_stream);
+  ET_CUDA0(cudaGetLastError());
+  return ET_OK;
+}
+
+et_status et_gather_tokens(const float* x_dev, const unsigned char* keep_dev, int N, int L, int D, const float* ln_g_dev,
+                           const float* ln_b_dev, float ln_eps, float* tokens_dev, size_t tokens_capacity_rows,
+                           int* frame_offsets_dev, int* token_pos_dev, int* n_tokens_host, void* cuda_stream) {
+  if (!x_dev || !keep_dev || !tokens_dev || !frame_offsets_dev || !token_pos_dev || !n_tokens_host) return ET_ERR_INVALID_ARG;
+  if ((ln_g_dev == nullptr) != (ln_b_dev == nullptr)) return ET_ERR_INVALID_ARG;
+  if (N < 1 || N > 65535 || L < 1 || L > 4096 || D < 4 || D % 4 != 0 || D > ROW_MAX_D) return ET_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  int* scratch = nullptr;
+  ET_CUDA0(cudaMalloc(&scratch, sizeof(int) * ((size_t)N + 2)));
+  int* count = scratch + 2;
+  launch_count_keep(keep_dev, N, L, count, nullptr, s);
+  launch_scan_counts(count, frame_offsets_dev, scratch, N, nullptr, s);
+  int totals[2] = {0, 0};
+  cudaError_t err = cudaMemcpyAsync(totals, scratch, sizeof(totals), cudaMemcpyDeviceToHost, s);
+  if (err == cudaSuccess) err = cudaStreamSynchronize(s);
+  if (err != cudaSuccess) { cudaFree(scratch); return ET_ERR_CUDA; }
+  if ((size_t)totals[1] > tokens_capacity_rows) { cudaFree(scratch); return ET_ERR_CAPACITY; }
+  launch_gather_tokens(x_dev, keep_dev, frame_offsets_dev, N, L, D, ln_g_dev, ln_b_dev, ln_eps, tokens_dev, token_pos_dev,
+                       nullptr, s);
+  err = cudaStreamSynchronize(s);
+  cudaFree(scratch);
+  if (err != cudaSuccess) return ET_ERR_CUDA;
+  *n_tokens_host = totals[1];
+  return ET_OK;
+}
+
+et_status et_linear_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, void* c_dev, int M, int N, int K,
+                         int epilogue, int gelu_tanh, const float* table_dev, int table_rows, int* status_dev,
+                         void* cuda_stream) {
+  if (!a_dev || !w_dev || !bias_dev || !c_dev) return ET_ERR_INVALID_ARG;
+  if (M < 1 || N < 8 || N % 8 != 0 || K < 8 || K % 8 != 0) return ET_ERR_SHAPE;
+  if (epilogue < 0 || epilogue > 3 || (epilogue == 3 && (!table_dev || table_rows < 1))) return ET_ERR_INVALID_ARG;
+  TmaDesc da, dw;
+  const char* err = nullptr;
+  if (!make_tma_2d_bf16(&da, a_dev, M, K, 128, &err) || !make_tma_2d_bf16(&dw, w_dev, N, K, gemm_bf16_pick_bn(N), &err))
+    return ET_ERR_CUDA;
+  ET_CUDA0(launch_gemm_bf16(da, dw, bias_dev, c_dev, M, N, K, epilogue, gelu_tanh, table_dev, table_rows, nullptr, 1,
+                            status_dev, (cudaStream_t)cuda_stream));
+  return ET_OK;
+}
+
+et_status et_attention(const void* qkv_dev, void* out_dev, float* lse_dev, int n, int L, int heads, int head_dim,
+                       int dtype, void* cuda_stream) {
+  if (!qkv_dev || !out_dev || !lse_dev) return ET_ERR_INVALID_ARG;
+  if (n < 1 || n > 65535 || L < 1 || heads < 1 || heads > 65535 || head_dim < 1 || head_dim > 128) return ET_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  if (dtype == ET_BF16) {
+    if (head_dim % 8 != 0) return ET_ERR_SHAPE;
+    launch_attention_bf16((const bf16*)qkv_dev, (bf16*)out_dev, lse_dev, n, L, heads, head_dim, nullptr, s);
+  } else if (dtype == ET_F32) {
+    launch_attention_f32((const float*)qkv_dev, (float*)out_dev, lse_dev, n, L, heads, head_dim, nullptr, s);
+  } else {
+    return ET_ERR_INVALID_ARG;
+  }
+  ET_CUDA0(cudaGetLastError());
+  return ET_OK;
+}
+
+et_status et_attention_scores(const void* qkv_dev, const float* lse_dev, float* partial_dev, float* score_dev, int n, int L,
+                              int heads, int head_dim, int dtype, void* cuda_stream) {
+  if (!qkv_dev || !lse_dev || !partial_dev || !score_dev) return ET_ERR_INVALID_ARG;
+  if (n < 1 || n > 65535 || L < 1 || heads < 1 || heads > 65535 || head_dim < 1 || head_dim > 128) return ET_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  if (dtype == ET_BF16) {
+    if (head_dim % 8 != 0) return ET_ERR_SHAPE;
+    launch_attention_scores_bf16((const bf16*)qkv_dev, lse_dev, partial_dev, score_dev, n, L, heads, head_dim, nullptr, s);
+  } else if (dtype == ET_F32) {
+    launch_attention_scores_f32((const float*)qkv_dev, lse_dev, partial_dev, score_dev, n, L, heads, head_dim, nullptr, s);
+  } else {
+    return ET_ERR_INVALID_ARG;
+  }
+  ET_CUDA0(cudaGetLastError());
+  return ET_OK;
+}
+
+et_status et_layernorm(const float* x_dev, const float* g_dev, const float* b_dev, float eps, void* y_dev, int rows, int D,
+                       int dtype, void* cuda_stream) {
+  if (!x_dev || !g_dev || !b_dev || !y_dev) return ET_ERR_INVALID_ARG;
+  if (rows < 1 || D < 4 || D % 4 != 0 || D > ROW_MAX_D) return ET_ERR_SHAPE;
+  if (dtype != ET_F32 && dtype != ET_BF16) return ET_ERR_INVALID_ARG;
+  launch_layernorm(x_dev, g_dev, b_dev, eps, y_dev, rows, D, dtype == ET_BF16, nullptr, 1, (cudaStream_t)cuda_stream);
+  ET_CUDA0(cudaGetLastError());
+  return ET_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,228 @@
+// Stage II kernels: per-frame amounts (Eq. 5-6), decoupled selection (Eq. 4 / Eq. 6), the scan of
+// the per-frame counts and the gather of the kept rows with warp-level prefix-sum compaction (Eq. 7).
+#include "common.cuh"
+#include "rowops.cuh"
+
+namespace et {
+
+// ---------------------------------------------------------------------------------------------
+// Per-video amounts and per-frame flags.  One thread per video computes k (Eq. 5 read as a
+// per-frame token count) and the window width w (Eq. 6) in double, with the same expression
+// order as a plain host evaluation; then all threads fill the per-frame arrays.
+// ---------------------------------------------------------------------------------------------
+__global__ void select_setup_kernel(SelectSetupArgs a) {
+  const int V = a.n_videos;
+  for (int v = threadIdx.x; v < V; v += blockDim.x) {
+    const int N = a.fl.vid_off[v + 1] - a.fl.vid_off[v];
+    const int B = a.orig_vid_off[v + 1] - a.orig_vid_off[v];
+    int k;
+    if (a.retain_mode == 1) k = (int)floor(a.retain * (double)B * (double)a.L / (double)max(N, 1) + 1e-9);
+    else k = (int)floor(a.retain * (double)a.L + 1e-9);
+    k = max(1, min(a.L, k));
+    const int w = max(1, a.L / k);
+    a.video_k[v] = k;
+    a.video_w[v] = w;
+  }
+  __syncthreads();
+  for (int v = 0; v < V; ++v) {
+    const int g0 = a.fl.vid_off[v], g1 = a.fl.vid_off[v + 1];
+    for (int t = g0 + threadIdx.x; t < g1; t += blockDim.x) {
+      const bool dyn = a.fl.role[t] != 1;
+      a.dynamic[t] = dyn ? 1 : 0;
+      a.k_frame[t] = a.video_k[v];
+      a.w_frame[t] = a.video_w[v];
+    }
+  }
+}
+
+void launch_select_setup(const SelectSetupArgs& a, int n_cap, cudaStream_t s) {
+  (void)n_cap;
+  ET_COUNT_LAUNCH();
+  select_setup_kernel<<<1, 256, 0, s>>>(a);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Selection: one CTA per frame, scores in shared memory.
+//   dynamic frame: token j is kept iff fewer than k tokens precede it in the order
+//                  (score descending, index ascending)  -> exact rank counting, O(L^2 / threads);
+//   static frame : the first maximum of each window of width w.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+select_tokens_kernel(const float* __restrict__ scores, const unsigned char* __restrict__ dynamic,
+                     const int* __restrict__ k_frame, const int* __restrict__ w_frame, int n_cap, int L,
+                     int selection_all, unsigned char* __restrict__ keep, int* __restrict__ count,
+                     const int* __restrict__ n_frames_dev) {
+  extern __shared__ float sh_a[];
+  const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
+  const int f = blockIdx.x;
+  if (f >= n) return;
+  const float* a = scores + (size_t)f * L;
+  unsigned char* kp = keep + (size_t)f * L;
+  if (selection_all) {
+    for (int j = threadIdx.x; j < L; j += blockDim.x) kp[j] = 1;
+    if (threadIdx.x == 0) count[f] = L;
+    return;
+  }
+  for (int j = threadIdx.x; j < L; j += blockDim.x) sh_a[j] = a[j];
+  __syncthreads();
+  if (dynamic[f]) {
+    const int k = k_frame[f];
+    for (int j = threadIdx.x; j < L; j += blockDim.x) {
+      const float aj = sh_a[j];
+      int rank = 0;
+      for (int i = 0; i < L; ++i) {
+        const float ai = sh_a[i];
+        rank += (ai > aj || (ai == aj && i < j)) ? 1 : 0;
+      }
+      kp[j] = rank < k ? 1 : 0;
+    }
+    if (threadIdx.x == 0) count[f] = min(k, L);
+  } else {
+    const int w = w_frame[f];
+    const int M = (L + w - 1) / w;
+    for (int j = threadIdx.x; j < L; j += blockDim.x) kp[j] = 0;
+    __syncthreads();
+    for (int m = threadIdx.x; m < M; m += blockDim.x) {
+      const int lo = m * w, hi = min(lo + w, L);
+      int best = lo;
+      for (int j = lo + 1; j < hi; ++j)
+        if (sh_a[j] > sh_a[best]) best = j;
+      kp[best] = 1;
+    }
+    if (threadIdx.x == 0) count[f] = M;
+  }
+}
+
+void launch_select_tokens(const float* scores, const unsigned char* dynamic, const int* k_frame, const int* w_frame,
+                          int n_cap, int L, int selection_all, unsigned char* keep, int* count,
+                          const int* n_frames_dev, cudaStream_t s) {
+  if (n_cap <= 0) return;
+  ET_COUNT_LAUNCH();
+  select_tokens_kernel<<<n_cap, 256, sizeof(float) * L, s>>>(scores, dynamic, k_frame, w_frame, n_cap, L,
+                                                             selection_all, keep, count, n_frames_dev);
+}
+
+// count[f] = number of set bytes of keep[f][:] (used when the mask is given, not decided)
+__global__ void count_keep_kernel(const unsigned char* __restrict__ keep, int n_cap, int L, int* __restrict__ count,
+                                  const int* __restrict__ n_frames_dev) {
+  const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
+  const int f = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (f >= n) return;
+  const int lane = threadIdx.x & 31;
+  int c = 0;
+  for (int j = lane; j < L; j += 32) c += keep[(size_t)f * L + j] ? 1 : 0;
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+  if (lane == 0) count[f] = c;
+}
+
+void launch_count_keep(const unsigned char* keep, int n_cap, int L, int* count, const int* n_frames_dev, cudaStream_t s) {
+  if (n_cap <= 0) return;
+  ET_COUNT_LAUNCH();
+  count_keep_kernel<<<cdiv(n_cap, 4), 128, 0, s>>>(keep, n_cap, L, count, n_frames_dev);
+}
+
+// Exclusive scan of the per-frame counts by one CTA (warp-shuffle scan + carry across chunks).
+__global__ void __launch_bounds__(1024)
+scan_counts_kernel(const int* __restrict__ count, int* __restrict__ frame_offsets, int* __restrict__ totals, int n_cap,
+                   const int* __restrict__ n_frames_dev) {
+  __shared__ int warp_tot[32];
+  __shared__ int carry;
+  const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int base = 0; base < n; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    const int v = i < n ? count[i] : 0;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += u;
+    }
+    if (lane == 31) warp_tot[wid] = inc;
+    __syncthreads();
+    if (wid == 0) {
+      int w = lane < (blockDim.x >> 5) ? warp_tot[lane] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, w, o);
+        if (lane >= o) w += u;
+      }
+      warp_tot[lane] = w;     // inclusive scan of warp totals
+    }
+    __syncthreads();
+    const int before = carry + (wid > 0 ? warp_tot[wid - 1] : 0) + inc - v;
+    if (i < n) frame_offsets[i] = before;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry += warp_tot[(blockDim.x >> 5) - 1];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    frame_offsets[n] = carry;
+    totals[0] = n;
+    totals[1] = carry;
+  }
+}
+
+void launch_scan_counts(const int* count, int* frame_offsets, int* totals, int n_cap, const int* n_frames_dev,
+                        cudaStream_t s) {
+  ET_COUNT_LAUNCH();
+  scan_counts_kernel<<<1, 1024, 0, s>>>(count, frame_offsets, totals, n_cap, n_frames_dev);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Gather (Eq. 7) with optional LayerNorm.  grid = (slices, frames).  Each CTA recomputes the
+// frame's compaction map by a warp-level prefix sum over ballots of the keep bytes (32 positions
+// per step, carry in a register), then its warps move their share of the kept rows:
+// warp-per-row, row in registers, LayerNorm statistics by shuffles.
+// ---------------------------------------------------------------------------------------------
+constexpr int GATHER_MAX_L = 4096;
+
+__global__ void __launch_bounds__(256)
+gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restrict__ keep,
+                     const int* __restrict__ frame_offsets, int n_cap, int L, int D, const float* __restrict__ ln_g,
+                     const float* __restrict__ ln_b, float eps, float* __restrict__ tokens,
+                     int* __restrict__ token_pos, const int* __restrict__ n_frames_dev) {
+  extern __shared__ unsigned short sh_pos[];   // [L] position of the r-th kept token of this frame
+  __shared__ int sh_kept;
+  const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
+  const int f = blockIdx.y;
+  if (f >= n) return;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const unsigned char* kp = keep + (size_t)f * L;
+  if (wid == 0) {
+    int carry = 0;
+    for (int base = 0; base < L; base += 32) {
+      const int j = base + lane;
+      const bool k = j < L && kp[j] != 0;
+      const unsigned m = __ballot_sync(0xffffffffu, k);
+      if (k) sh_pos[carry + __popc(m & ((1u << lane) - 1u))] = (unsigned short)j;
+      carry += __popc(m);
+    }
+    if (lane == 0) sh_kept = carry;
+  }
+  __syncthreads();
+  const int kept = sh_kept;
+  const int out0 = frame_offsets[f];
+  for (int r = blockIdx.x * nwarps + wid; r < kept; r += gridDim.x * nwarps) {
+    const int j = sh_pos[r];
+    float4 v[ROW_MAX_VEC];
+    load_row(x + ((size_t)f * L + j) * D, D, lane, v);
+    if (ln_g) layernorm_row_inplace(v, D, lane, ln_g, ln_b, eps);
+    store_row<float>(tokens + (size_t)(out0 + r) * D, D, lane, v);
+    if (lane == 0) token_pos[out0 + r] = j;
+  }
+}
+
+void launch_gather_tokens(const float* x, const unsigned char* keep, const int* frame_offsets, int n_cap, int L, int D,
+                          const float* ln_g, const float* ln_b, float eps, float* tokens, int* token_pos,
+                          const int* n_frames_dev, cudaStream_t s) {
+  if (n_cap <= 0) return;
+  const int slices = max(1, min(16, cdiv(L, 64)));
+  ET_COUNT_LAUNCH();
+  gather_tokens_kernel<<<dim3(slices, n_cap), 256, sizeof(unsigned short) * L, s>>>(
+      x, keep, frame_offsets, n_cap, L, D, ln_g, ln_b, eps, tokens, token_pos, n_frames_dev);
+}
+
+}  // namespace et
