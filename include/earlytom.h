@@ -175,6 +175,34 @@ ET_API void et_destroy(et_encoder* enc);
 ET_API const char* et_status_string(et_status s);
 ET_API const char* et_last_error(const et_encoder* enc); /* text of the last failure on this encoder */
 
+/* Per-category device timings of the encode calls (no counterpart in the paper: measurement aid).
+ * While enabled, every encode call brackets its kernel groups with CUDA events on the call's
+ * stream and, after its final synchronisation, adds the elapsed times and the algorithmic work
+ * (FLOPs for the tensor-core categories, bytes for the bandwidth categories, computed from the
+ * frame counts the call actually ran with) to the counters. */
+enum {
+  ET_CAT_IM2COL = 0,    /* bytes: frames read + patch matrix written */
+  ET_CAT_GEMM = 1,      /* flops: 2*M*N*K of every dense layer (patch embed, QKV, out-proj, MLP) */
+  ET_CAT_ATTENTION = 2, /* flops: 4*L*L*D per frame per block */
+  ET_CAT_LAYERNORM = 3, /* bytes: rows*D*(4 + output element size) */
+  ET_CAT_SIMILARITY = 4,/* bytes: n*L*D*4 read once + cosines written and re-read */
+  ET_CAT_PLAN = 5,      /* bytes: 0 (latency-bound scalar work) */
+  ET_CAT_MERGE = 6,     /* bytes: source frames read + output frames written */
+  ET_CAT_SCORES = 7,    /* flops: 2*L*L*D per output frame */
+  ET_CAT_SELECT = 8,    /* bytes: scores read + mask written */
+  ET_CAT_GATHER = 9,    /* bytes: kept rows read + written */
+  ET_PROF_CATS = 10
+};
+typedef struct {
+  double ms[ET_PROF_CATS];
+  double work[ET_PROF_CATS];
+  unsigned long long launches[ET_PROF_CATS];
+  int calls;
+} et_profile;
+/* on != 0: reset the counters and start collecting; 0: stop. */
+ET_API et_status et_profile_enable(et_encoder* enc, int on);
+ET_API et_status et_profile_read(const et_encoder* enc, et_profile* out);
+
 /* Number of kernels the library has launched in this process (all encoders); for benchmarks. */
 ET_API unsigned long long et_kernel_launch_count(void);
 

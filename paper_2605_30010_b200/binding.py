@@ -20,7 +20,7 @@ ET_MAX_MERGE_LAYERS = 8
 STATUS_NAMES = ["ET_OK", "ET_ERR_INVALID_ARG", "ET_ERR_SHAPE", "ET_ERR_CAPACITY", "ET_ERR_OOM", "ET_ERR_CUDA",
                 "ET_ERR_TIMEOUT", "ET_ERR_WEIGHTS"]
 EXPORTS = ["et_encoder_create", "et_encode_video", "et_encode_batch", "et_encode_batch_host", "et_destroy",
-           "et_status_string", "et_last_error", "et_kernel_launch_count", "et_frame_similarity", "et_merge_plan",
+           "et_status_string", "et_last_error", "et_kernel_launch_count", "et_profile_enable", "et_profile_read", "et_frame_similarity", "et_merge_plan",
            "et_merge_frames", "et_select_tokens", "et_gather_tokens", "et_linear_bf16", "et_attention",
            "et_attention_scores", "et_layernorm"]
 
@@ -81,6 +81,15 @@ class et_host_buffers(C.Structure):
                 ("video_frame_offsets", C.c_void_p), ("capacity_tokens", C.c_size_t), ("capacity_frames", C.c_size_t)]
 
 
+ET_PROF_CATS = 10
+PROF_NAMES = ["im2col", "gemm", "attention", "layernorm", "similarity", "plan", "merge", "scores", "select", "gather"]
+
+
+class et_profile(C.Structure):
+    _fields_ = [("ms", C.c_double * ET_PROF_CATS), ("work", C.c_double * ET_PROF_CATS),
+                ("launches", C.c_ulonglong * ET_PROF_CATS), ("calls", C.c_int)]
+
+
 def load_library(path: str = _LIB_PATH) -> C.CDLL:
     if not os.path.exists(path):
         raise ImportError(f"{path} is missing: build it with `python -m paper_2605_30010_b200.build` "
@@ -102,6 +111,8 @@ def load_library(path: str = _LIB_PATH) -> C.CDLL:
     lib.et_last_error.restype = C.c_char_p
     lib.et_kernel_launch_count.argtypes = []
     lib.et_kernel_launch_count.restype = C.c_ulonglong
+    lib.et_profile_enable.argtypes = [vp, i]
+    lib.et_profile_read.argtypes = [vp, C.POINTER(et_profile)]
     lib.et_frame_similarity.argtypes = [vp, i, i, i, vp, vp, vp]
     lib.et_merge_plan.argtypes = [vp, vp, i, i, d, d, d, i, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.et_merge_frames.argtypes = [vp, vp, i, i, vp, vp, vp, vp, vp, vp]
@@ -374,6 +385,19 @@ def et_encode_batch_host(enc: Encoder, frames_host, video_offsets: Sequence[int]
 
 def et_kernel_launch_count() -> int:
     return int(lib().et_kernel_launch_count())
+
+
+def et_profile_enable(enc: Encoder, on: bool) -> None:
+    _check(lib().et_profile_enable(enc.handle, 1 if on else 0))
+
+
+def et_profile_read(enc: Encoder) -> dict:
+    """{category: {"ms", "work", "launches"}} accumulated since et_profile_enable(enc, True), plus "calls"."""
+    p = et_profile()
+    _check(lib().et_profile_read(enc.handle, C.byref(p)))
+    out = {PROF_NAMES[i]: {"ms": p.ms[i], "work": p.work[i], "launches": int(p.launches[i])} for i in range(ET_PROF_CATS)}
+    out["calls"] = p.calls
+    return out
 
 
 # ---- single steps (torch CUDA tensors in, torch CUDA tensors out) ---------------------------

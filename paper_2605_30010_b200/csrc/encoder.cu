@@ -93,6 +93,13 @@ struct et_encoder {
   float* h_scores = nullptr;
   unsigned char* h_keep = nullptr;
   int* h_video_kw = nullptr;                   // [2*Vmax]
+  // profiling
+  bool prof_on = false;
+  et_profile prof{};
+  std::vector<cudaEvent_t> prof_events;
+  struct Span { int cat; int ev; unsigned long long launches0, launches1; };
+  std::vector<Span> prof_spans;
+  size_t prof_next_event = 0;
 };
 
 namespace {
@@ -101,6 +108,33 @@ et_status fail(et_encoder* e, et_status st, const std::string& msg) {
   if (e) e->last_error = msg;
   return st;
 }
+
+void prof_begin(et_encoder* e, int cat, cudaStream_t s) {
+  if (!e->prof_on) return;
+  if (e->prof_next_event + 2 > e->prof_events.size()) {
+    for (int i = 0; i < 2; ++i) {
+      cudaEvent_t ev;
+      if (cudaEventCreate(&ev) != cudaSuccess) return;
+      e->prof_events.push_back(ev);
+    }
+  }
+  et_encoder::Span sp{cat, (int)e->prof_next_event, g_kernel_launches.load(), 0};
+  cudaEventRecord(e->prof_events[e->prof_next_event], s);
+  e->prof_next_event += 2;
+  e->prof_spans.push_back(sp);
+}
+void prof_end(et_encoder* e, cudaStream_t s) {
+  if (!e->prof_on || e->prof_spans.empty()) return;
+  et_encoder::Span& sp = e->prof_spans.back();
+  sp.launches1 = g_kernel_launches.load();
+  cudaEventRecord(e->prof_events[sp.ev + 1], s);
+}
+#define PROF(cat, ...)        \
+  do {                        \
+    prof_begin(e, (cat), s);  \
+    __VA_ARGS__;              \
+    prof_end(e, s);           \
+  } while (0)
 
 #define ET_CUDA(e, call)                                                                        \
   do {                                                                                          \
@@ -227,21 +261,23 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
       ET_CUDA(e, cudaMemcpyAsync(e->forced_mrg[i], hm, fp->n_in[i], cudaMemcpyHostToDevice, s));
     }
   }
+  e->prof_spans.clear();
+  e->prof_next_event = 0;
   int lst = 0, cur = 0;
   launch_init_frames(e->fl[0], e->orig_vid_off, V, T, s);
 
   // patch embedding: im2col + dense layer with the position table added in the epilogue
-  launch_im2col(frames_dev, e->Pm, T, c.image_size, c.patch_size, e->Kp, e->bf, nullptr, s);
-  ET_TRY(dense(e, e->Pm, e->d_Pm, W + e->off_patch_w, e->d_patch_w, W + e->off_patch_b, e->X[cur], rows_cap, D,
-               e->bf ? e->Kp : e->P, EPI_TABLE, W + e->off_pos, L, nullptr, s));
+  PROF(ET_CAT_IM2COL, launch_im2col(frames_dev, e->Pm, T, c.image_size, c.patch_size, e->Kp, e->bf, nullptr, s));
+  PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Pm, e->d_Pm, W + e->off_patch_w, e->d_patch_w, W + e->off_patch_b, e->X[cur], rows_cap, D,
+               e->bf ? e->Kp : e->P, EPI_TABLE, W + e->off_pos, L, nullptr, s)));
 
   int mi = 0;
   for (int layer = 0; layer < c.num_layers; ++layer) {
     if (mi < p->num_merge_layers && p->merge_layers[mi] == layer) {
       // Stage I at this block: similarities -> plan -> weighted merge + compaction
       const int* n_dev = e->fl[lst].n;
-      launch_token_cosines(e->X[cur], e->cosbuf, T, L, D, n_dev, s);
-      launch_reduce_cosines(e->cosbuf, e->simbuf, T, L, n_dev, s);
+      PROF(ET_CAT_SIMILARITY, launch_token_cosines(e->X[cur], e->cosbuf, T, L, D, n_dev, s));
+      PROF(ET_CAT_SIMILARITY, launch_reduce_cosines(e->cosbuf, e->simbuf, T, L, n_dev, s));
       PlanArgs a{};
       a.sim = e->simbuf; a.cur = e->fl[lst]; a.nxt = e->fl[lst ^ 1]; a.plan = e->plan; a.trace = e->tr[mi];
       a.forced_seg_start = fp ? e->forced_seg[mi] : nullptr;
@@ -250,60 +286,64 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
       a.alpha = p->ema_alpha; a.tau_seg = p->tau_seg; a.tau_merge = p->tau_merge;
       a.weighted = p->weighted_merge; a.allow_merge = 1; a.n_videos = V;
       a.n_hist_slot = e->d_small + 2 + mi; a.status = e->d_small + 10;
-      launch_merge_plan(a, s);
-      launch_merge_frames(e->X[cur], e->X[cur ^ 1], T, L * D, e->fl[lst ^ 1].n, e->plan, s);
+      PROF(ET_CAT_PLAN, launch_merge_plan(a, s));
+      PROF(ET_CAT_MERGE, launch_merge_frames(e->X[cur], e->X[cur ^ 1], T, L * D, e->fl[lst ^ 1].n, e->plan, s));
       cur ^= 1; lst ^= 1; ++mi;
     }
     const int* n_dev = e->fl[lst].n;
     const LayerOffsets& o = e->lo[layer];
     const LayerBf16* b = e->bf ? &e->lb[layer] : nullptr;
     static const TmaDesc none{};
-    launch_layernorm(e->X[cur], W + o.ln1_g, W + o.ln1_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s);
-    ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.wqkv, b ? b->d_wqkv : none, W + o.bqkv, e->QKV, rows_cap, 3 * D, D, EPI_STORE,
-                 nullptr, 1, n_dev, s));
-    if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, s);
-    else launch_attention_f32((const float*)e->QKV, (float*)e->O, e->lse, T, L, H, dh, n_dev, s);
+    PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln1_g, W + o.ln1_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
+    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.wqkv, b ? b->d_wqkv : none, W + o.bqkv, e->QKV, rows_cap, 3 * D, D, EPI_STORE,
+                 nullptr, 1, n_dev, s)));
+    PROF(ET_CAT_ATTENTION, {
+      if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, s);
+      else launch_attention_f32((const float*)e->QKV, (float*)e->O, e->lse, T, L, H, dh, n_dev, s);
+    });
     if (layer == c.num_layers - 1) {
-      if (e->bf) launch_attention_scores_bf16((const bf16*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
-      else launch_attention_scores_f32((const float*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
+      PROF(ET_CAT_SCORES, {
+        if (e->bf) launch_attention_scores_bf16((const bf16*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
+        else launch_attention_scores_f32((const float*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
+      });
     }
-    ET_TRY(dense(e, e->O, e->d_O, W + o.wo, b ? b->d_wo : none, W + o.bo, e->X[cur], rows_cap, D, D, EPI_RESIDUAL,
-                 nullptr, 1, n_dev, s));
-    launch_layernorm(e->X[cur], W + o.ln2_g, W + o.ln2_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s);
-    ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, W + o.b1, e->Hm, rows_cap, Mlp, D, EPI_GELU, nullptr, 1,
-                 n_dev, s));
-    ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, W + o.b2, e->X[cur], rows_cap, D, Mlp, EPI_RESIDUAL,
-                 nullptr, 1, n_dev, s));
+    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->O, e->d_O, W + o.wo, b ? b->d_wo : none, W + o.bo, e->X[cur], rows_cap, D, D, EPI_RESIDUAL,
+                 nullptr, 1, n_dev, s)));
+    PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln2_g, W + o.ln2_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
+    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, W + o.b1, e->Hm, rows_cap, Mlp, D, EPI_GELU, nullptr, 1,
+                 n_dev, s)));
+    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, W + o.b2, e->X[cur], rows_cap, D, Mlp, EPI_RESIDUAL,
+                 nullptr, 1, n_dev, s)));
   }
   const int* n_dev = e->fl[lst].n;
   if (p->num_merge_layers == 0) {
     // Stage I off: the segment list of Stage II comes from the streaming segmentation of the final features
-    launch_token_cosines(e->X[cur], e->cosbuf, T, L, D, n_dev, s);
-    launch_reduce_cosines(e->cosbuf, e->simbuf, T, L, n_dev, s);
+    PROF(ET_CAT_SIMILARITY, launch_token_cosines(e->X[cur], e->cosbuf, T, L, D, n_dev, s));
+    PROF(ET_CAT_SIMILARITY, launch_reduce_cosines(e->cosbuf, e->simbuf, T, L, n_dev, s));
     PlanArgs a{};
     a.sim = e->simbuf; a.cur = e->fl[lst]; a.nxt = e->fl[lst ^ 1]; a.plan = e->plan; a.trace = e->tr[0];
     a.alpha = p->ema_alpha; a.tau_seg = p->tau_seg; a.tau_merge = p->tau_merge;
     a.weighted = p->weighted_merge; a.allow_merge = 0; a.n_videos = V; a.status = e->d_small + 10;
-    launch_merge_plan(a, s);
+    PROF(ET_CAT_PLAN, launch_merge_plan(a, s));
   }
   // Stage II
   SelectSetupArgs sa{};
   sa.fl = e->fl[lst]; sa.orig_vid_off = e->orig_vid_off; sa.n_videos = V; sa.L = L; sa.selection = p->selection;
   sa.retain_mode = p->retain_mode; sa.retain = p->retain; sa.dynamic = e->dynamic; sa.k_frame = e->k_frame;
   sa.w_frame = e->w_frame; sa.video_k = e->video_k; sa.video_w = e->video_w;
-  launch_select_setup(sa, T, s);
+  PROF(ET_CAT_SELECT, launch_select_setup(sa, T, s));
   if (fp && fp->keep) {
     memcpy(e->h_keep_stage, fp->keep, (size_t)fp->n_final * L);
     ET_CUDA(e, cudaMemcpyAsync(e->keep, e->h_keep_stage, (size_t)fp->n_final * L, cudaMemcpyHostToDevice, s));
-    launch_count_keep(e->keep, T, L, e->count, n_dev, s);
+    PROF(ET_CAT_SELECT, launch_count_keep(e->keep, T, L, e->count, n_dev, s));
   } else {
     if (p->selection == 2) ET_CUDA(e, cudaMemsetAsync(e->dynamic, 1, T, s));   // plain top-k: every frame ranks globally
-    launch_select_tokens(e->scores, e->dynamic, e->k_frame, e->w_frame, T, L, p->selection == 0, e->keep, e->count, n_dev, s);
-    if (p->selection == 2) launch_select_setup(sa, T, s);                      // restore the reported dynamic flags
+    PROF(ET_CAT_SELECT, launch_select_tokens(e->scores, e->dynamic, e->k_frame, e->w_frame, T, L, p->selection == 0, e->keep, e->count, n_dev, s));
+    if (p->selection == 2) PROF(ET_CAT_SELECT, launch_select_setup(sa, T, s));                      // restore the reported dynamic flags
   }
-  launch_scan_counts(e->count, e->frame_offsets, e->d_small, T, n_dev, s);
-  launch_gather_tokens(e->X[cur], e->keep, e->frame_offsets, T, L, D, c.post_layernorm ? W + e->off_post_g : nullptr,
-                       c.post_layernorm ? W + e->off_post_b : nullptr, c.ln_eps, e->tokens, e->token_pos, n_dev, s);
+  PROF(ET_CAT_SELECT, launch_scan_counts(e->count, e->frame_offsets, e->d_small, T, n_dev, s));
+  PROF(ET_CAT_GATHER, launch_gather_tokens(e->X[cur], e->keep, e->frame_offsets, T, L, D, c.post_layernorm ? W + e->off_post_g : nullptr,
+                       c.post_layernorm ? W + e->off_post_b : nullptr, c.ln_eps, e->tokens, e->token_pos, n_dev, s));
   ET_CUDA(e, cudaMemcpyAsync(e->h_small, e->d_small, sizeof(int) * 16, cudaMemcpyDeviceToHost, s));
   ET_CUDA(e, cudaGetLastError());
   ET_CUDA(e, cudaStreamSynchronize(s));
@@ -326,6 +366,36 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
       if (m < p->num_merge_layers && p->merge_layers[m] == layer) { alive = e->h_small[2 + m]; ++m; }
       r.frames_per_block[layer] = alive;
     }
+  }
+  if (e->prof_on) {
+    for (const et_encoder::Span& sp : e->prof_spans) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, e->prof_events[sp.ev], e->prof_events[sp.ev + 1]) == cudaSuccess) e->prof.ms[sp.cat] += ms;
+      e->prof.launches[sp.cat] += sp.launches1 - sp.launches0;
+    }
+    // algorithmic work of this call from the frame counts it actually ran with
+    const double dL = L, dD = D, dM = Mlp, es = e->bf ? 2.0 : 4.0;
+    double* wk = e->prof.work;
+    wk[ET_CAT_IM2COL] += (double)T * 3.0 * c.image_size * c.image_size * 4.0 + (double)T * dL * e->Kp * es;
+    wk[ET_CAT_GEMM] += 2.0 * T * dL * dD * e->P;
+    int n_in = T;
+    for (int layer = 0, m = 0; layer < c.num_layers; ++layer) {
+      if (m < p->num_merge_layers && p->merge_layers[m] == layer) {
+        const int n_out = e->h_small[2 + m];
+        wk[ET_CAT_SIMILARITY] += (double)n_in * dL * dD * 4.0 + 2.0 * (n_in - 1) * dL * 4.0;
+        wk[ET_CAT_MERGE] += ((double)n_in + n_out) * dL * dD * 4.0;
+        n_in = n_out; ++m;
+      }
+      const double rows = (double)r.frames_per_block[layer] * dL;
+      wk[ET_CAT_GEMM] += 2.0 * rows * (4.0 * dD * dD + 2.0 * dD * dM);
+      wk[ET_CAT_ATTENTION] += 4.0 * rows * dL * dD;
+      wk[ET_CAT_LAYERNORM] += 2.0 * rows * dD * (4.0 + es);
+    }
+    if (p->num_merge_layers == 0) wk[ET_CAT_SIMILARITY] += (double)N * dL * dD * 4.0 + 2.0 * (N - 1) * dL * 4.0;
+    wk[ET_CAT_SCORES] += 2.0 * N * dL * dL * dD;
+    wk[ET_CAT_SELECT] += (double)N * dL * 5.0;
+    wk[ET_CAT_GATHER] += 2.0 * n_tok * dD * 4.0;
+    e->prof.calls += 1;
   }
   if (p->want_trace) {
     et_trace& t = e->trace;
@@ -480,6 +550,7 @@ void et_destroy(et_encoder* e) {
   if (!e) return;
   for (void* p : e->dev_allocs) cudaFree(p);
   for (void* p : e->host_allocs) cudaFreeHost(p);
+  for (cudaEvent_t ev : e->prof_events) cudaEventDestroy(ev);
   delete e;
 }
 
@@ -540,6 +611,19 @@ const char* et_status_string(et_status s) {
 const char* et_last_error(const et_encoder* enc) { return enc ? enc->last_error.c_str() : ""; }
 
 unsigned long long et_kernel_launch_count(void) { return g_kernel_launches.load(); }
+
+et_status et_profile_enable(et_encoder* enc, int on) {
+  if (!enc) return ET_ERR_INVALID_ARG;
+  enc->prof_on = on != 0;
+  if (on) memset(&enc->prof, 0, sizeof(enc->prof));
+  return ET_OK;
+}
+
+et_status et_profile_read(const et_encoder* enc, et_profile* out) {
+  if (!enc || !out) return ET_ERR_INVALID_ARG;
+  *out = enc->prof;
+  return ET_OK;
+}
 
 // ------------------------------------------------------------------------------------------------
 // single steps
