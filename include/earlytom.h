@@ -219,6 +219,22 @@ ET_API unsigned long long et_kernel_launch_count(void);
 ET_API et_status et_frame_similarity(const float* x_dev, int n, int L, int D, float* cos_scratch_dev, float* sim_dev,
                               void* cuda_stream);
 
+/* The paper has no counterpart to this call: it is et_frame_similarity for callers that cannot
+ * allocate device memory (an allocator that already owns the whole card, a thread that may not
+ * take the device-wide synchronisation of cudaMalloc/cudaFree, a host that forbids allocation after
+ * start-up).  The per-position cosines go to a fixed 256 KiB array inside the library image
+ * instead of a caller buffer, so only x_dev (fp32 [n][L][D]) and sim_dev (fp32 [n-1]) are passed;
+ * same arithmetic, same reduction order, same results as et_frame_similarity.
+ *   - limit: (n-1)*L <= 65536, otherwise ET_ERR_CAPACITY and nothing is launched;
+ *   - the call itself never allocates or frees; every GPU that loads the library holds the array
+ *     until the process exits;
+ *   - the first call on each device looks up the array's device address (host-side, once); make
+ *     that first call before any stream capture begins;
+ *   - the array is shared by all calls and keeps the last call's cosines; nothing needs clearing
+ *     (every value read is written first), but calls that overlap on the GPU race on it. */
+ET_API et_status et_frame_similarity_static(const float* x_dev, int n, int L, int D, float* sim_dev,
+                                            void* cuda_stream);
+
 /* Paper Eq. 1-2 / Alg. 1 decisions for V videos from given similarities.  sim_dev [n] (entry t =
  * frames t,t+1; entries at video ends ignored), video_offsets_dev int [V+1].  Outputs (device):
  * seg_start [n], merge_next [n] bytes, ema [n] fp32, n_out int [1], and the plan of the merged

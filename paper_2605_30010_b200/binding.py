@@ -20,7 +20,8 @@ ET_MAX_MERGE_LAYERS = 8
 STATUS_NAMES = ["ET_OK", "ET_ERR_INVALID_ARG", "ET_ERR_SHAPE", "ET_ERR_CAPACITY", "ET_ERR_OOM", "ET_ERR_CUDA",
                 "ET_ERR_TIMEOUT", "ET_ERR_WEIGHTS"]
 EXPORTS = ["et_encoder_create", "et_encode_video", "et_encode_batch", "et_encode_batch_host", "et_destroy",
-           "et_status_string", "et_last_error", "et_kernel_launch_count", "et_profile_enable", "et_profile_read", "et_frame_similarity", "et_merge_plan",
+           "et_status_string", "et_last_error", "et_kernel_launch_count", "et_profile_enable", "et_profile_read",
+           "et_frame_similarity_static", "et_frame_similarity", "et_merge_plan",
            "et_merge_frames", "et_select_tokens", "et_gather_tokens", "et_linear_bf16", "et_attention",
            "et_attention_scores", "et_layernorm"]
 
@@ -114,6 +115,7 @@ def load_library(path: str = _LIB_PATH) -> C.CDLL:
     lib.et_profile_enable.argtypes = [vp, i]
     lib.et_profile_read.argtypes = [vp, C.POINTER(et_profile)]
     lib.et_frame_similarity.argtypes = [vp, i, i, i, vp, vp, vp]
+    lib.et_frame_similarity_static.argtypes = [vp, i, i, i, vp, vp]
     lib.et_merge_plan.argtypes = [vp, vp, i, i, d, d, d, i, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.et_merge_frames.argtypes = [vp, vp, i, i, vp, vp, vp, vp, vp, vp]
     lib.et_select_tokens.argtypes = [vp, vp, vp, vp, i, i, vp, vp, vp]
@@ -409,6 +411,18 @@ def et_frame_similarity(x, stream=None):
     sim = torch.zeros(max(n - 1, 1), dtype=torch.float32, device=x.device)
     _check(lib().et_frame_similarity(_ptr(x), n, L, D, _ptr(cosb), _ptr(sim), _stream_ptr(stream)))
     return sim[:n - 1], cosb[:n - 1]
+
+
+def et_frame_similarity_static(x, sim_out=None, stream=None):
+    """Adjacent-frame similarity without any allocation inside the library: the cosines go to the
+    library's built-in scratch array.  `sim_out` (float32 cuda [n-1]) is the caller's output buffer;
+    it is created here with torch only when the caller does not bring one."""
+    import torch
+    n, L, D = x.shape
+    if sim_out is None:
+        sim_out = torch.zeros(max(n - 1, 1), dtype=torch.float32, device=x.device)
+    _check(lib().et_frame_similarity_static(_ptr(x), n, L, D, _ptr(sim_out), _stream_ptr(stream)))
+    return sim_out[:n - 1]
 
 
 def et_merge_plan(sim, video_offsets, alpha, tau_seg, tau_merge, weighted=1, stream=None):

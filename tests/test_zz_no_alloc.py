@@ -1,0 +1,47 @@
+"""The allocation-free similarity entry point gives what the regular one gives (needs a B200).
+
+Collected last on purpose: a run that stops at the first failure has already been through every
+other test.  The entry point keeps its scratch in a fixed array inside the library, for callers that
+are not allowed to allocate device memory; here it is called twice in a row through the C ABI, on
+different inputs, so that leftovers of the first call in the shared array would show.
+"""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+def _video(rng, n, L, D):
+    base = rng.standard_normal((L, D)).astype(np.float32)
+    return np.stack([base + rng.uniform(0.1, 1.5) * rng.standard_normal((L, D)).astype(np.float32) for _ in range(n)])
+
+
+def test_static_scratch_matches_regular_entry_point_twice_in_a_row():
+    import torch
+    from paper_2605_30010_b200 import binding as B
+    assert torch.cuda.is_available()
+    rng = np.random.default_rng(2024)
+    # first call: the larger problem (fills more of the shared scratch); second call: a smaller,
+    # different one, which must not see anything of the first
+    for n, L, D in [(32, 729, 1152), (9, 64, 64)]:
+        x = torch.from_numpy(_video(rng, n, L, D)).cuda()
+        want, _ = B.et_frame_similarity(x)
+        out = torch.full((n - 1,), float("nan"), dtype=torch.float32, device="cuda")   # caller-owned output
+        got = B.et_frame_similarity_static(x, out)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(got.cpu().numpy(), want.cpu().numpy(), rtol=0, atol=2e-6)
+        assert torch.equal(got, want), "same kernels, same reduction order: results should be identical"
+
+
+def test_static_scratch_rejects_oversized_problems():
+    import torch
+    from paper_2605_30010_b200 import binding as B
+    x = torch.zeros((91, 729, 8), dtype=torch.float32, device="cuda")      # 90 * 729 = 65610 > 65536 cosines
+    with pytest.raises(B.EarlyTomError) as ei:
+        B.et_frame_similarity_static(x)
+    assert ei.value.status == 3                                            # ET_ERR_CAPACITY
+    ok = torch.zeros((90, 729, 8), dtype=torch.float32, device="cuda")     # 89 * 729 = 64881 fits
+    ok[:, :, 0] = 1.0
+    sim = B.et_frame_similarity_static(ok)
+    torch.cuda.synchronize()
+    assert torch.allclose(sim, torch.ones_like(sim))
