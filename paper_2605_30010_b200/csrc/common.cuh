@@ -72,12 +72,17 @@ struct TmaDesc { alignas(64) unsigned char bytes[128]; };
 // Build a 2-D bf16 tensor map: rows x cols (cols contiguous), box box_rows x 64 cols, 128-byte swizzle.
 bool make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
                       const char** err);
+// Tensor map of a dense layer's output c [rows][cols] (fp32 or bf16): 32 x 32 boxes for the epilogue's
+// TMA stores / reduce-adds.
+bool make_tma_out(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, bool fp32, const char** err);
 int gemm_bf16_pick_bn(int N);
-// c = epi(a[M][K] * w[N][K]^T + bias).  Descriptors must have been built for (a: M_cap x K, box 128)
-// and (w: N x K, box = gemm_bf16_pick_bn(N)).
-cudaError_t launch_gemm_bf16(const TmaDesc& da, const TmaDesc& dw, const float* bias, void* c, int M_cap, int N, int K,
-                             int epilogue, int gelu_tanh, const float* table, int table_rows, const int* n_frames_dev,
-                             int rows_per_frame, int* status_dev, cudaStream_t s);
+// Rows of the w box: each CTA of a pair loads half of the tile's BN weight rows.
+int gemm_bf16_w_box_rows(int N);
+// c = epi(a[M][K] * w[N][K]^T + bias).  Descriptors must have been built for (a: M_cap x K, box 128),
+// (w: N x K, box = gemm_bf16_w_box_rows(N)) and (c: make_tma_out; unused by EPI_TABLE).
+cudaError_t launch_gemm_bf16(const TmaDesc& da, const TmaDesc& dw, const TmaDesc& dc, const float* bias, void* c,
+                             int M_cap, int N, int K, int epilogue, int gelu_tanh, const float* table, int table_rows,
+                             const int* n_frames_dev, int rows_per_frame, int* status_dev, cudaStream_t s);
 
 // ---- attention_simt.cu / attention_mma.cu --------------------------------------------------
 void launch_attention_f32(const float* qkv, float* out, float* lse, int n_cap, int L, int heads, int dh,

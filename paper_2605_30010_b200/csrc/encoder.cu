@@ -65,7 +65,8 @@ struct et_encoder {
   // activations
   float* X[2] = {nullptr, nullptr};
   void *Pm = nullptr, *Xn = nullptr, *QKV = nullptr, *O = nullptr, *Hm = nullptr;
-  TmaDesc d_Pm, d_Xn, d_O, d_Hm;
+  TmaDesc d_Pm, d_Xn, d_O, d_Hm;                   // operand (A) maps
+  TmaDesc c_X[2], c_QKV, c_Hm;                      // output (C) maps
   float *lse = nullptr, *score_partial = nullptr, *scores = nullptr, *cosbuf = nullptr, *simbuf = nullptr;
   float* frames_stage = nullptr;               // device staging for the *_host entry point (lazy)
 
@@ -208,10 +209,10 @@ et_status validate_params(const et_encoder* e, const et_params* p) {
 
 // One dense layer of the encoder on the arithmetic path the encoder was created with.
 et_status dense(et_encoder* e, const void* a, const TmaDesc& da, const float* w_f32, const TmaDesc& dw,
-                const float* bias, void* c, int M_cap, int N, int K, int epi, const float* table, int table_rows,
+                const TmaDesc& dc, const float* bias, void* c, int M_cap, int N, int K, int epi, const float* table, int table_rows,
                 const int* n_dev, cudaStream_t s) {
   if (e->bf) {
-    ET_CUDA(e, launch_gemm_bf16(da, dw, bias, c, M_cap, N, K, epi, e->cfg.gelu_tanh, table, table_rows, n_dev, e->L,
+    ET_CUDA(e, launch_gemm_bf16(da, dw, dc, bias, c, M_cap, N, K, epi, e->cfg.gelu_tanh, table, table_rows, n_dev, e->L,
                                 e->d_small + 10, s));
   } else {
     launch_gemm_f32((const float*)a, w_f32, bias, (float*)c, M_cap, N, K, epi, e->cfg.gelu_tanh, table, table_rows,
@@ -268,7 +269,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
 
   // patch embedding: im2col + dense layer with the position table added in the epilogue
   PROF(ET_CAT_IM2COL, launch_im2col(frames_dev, e->Pm, T, c.image_size, c.patch_size, e->Kp, e->bf, nullptr, s));
-  PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Pm, e->d_Pm, W + e->off_patch_w, e->d_patch_w, W + e->off_patch_b, e->X[cur], rows_cap, D,
+  PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Pm, e->d_Pm, W + e->off_patch_w, e->d_patch_w, e->c_X[cur], W + e->off_patch_b, e->X[cur], rows_cap, D,
                e->bf ? e->Kp : e->P, EPI_TABLE, W + e->off_pos, L, nullptr, s)));
 
   int mi = 0;
@@ -295,7 +296,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     const LayerBf16* b = e->bf ? &e->lb[layer] : nullptr;
     static const TmaDesc none{};
     PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln1_g, W + o.ln1_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
-    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.wqkv, b ? b->d_wqkv : none, W + o.bqkv, e->QKV, rows_cap, 3 * D, D, EPI_STORE,
+    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.wqkv, b ? b->d_wqkv : none, e->c_QKV, W + o.bqkv, e->QKV, rows_cap, 3 * D, D, EPI_STORE,
                  nullptr, 1, n_dev, s)));
     PROF(ET_CAT_ATTENTION, {
       if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, s);
@@ -307,12 +308,12 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
         else launch_attention_scores_f32((const float*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
       });
     }
-    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->O, e->d_O, W + o.wo, b ? b->d_wo : none, W + o.bo, e->X[cur], rows_cap, D, D, EPI_RESIDUAL,
+    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->O, e->d_O, W + o.wo, b ? b->d_wo : none, e->c_X[cur], W + o.bo, e->X[cur], rows_cap, D, D, EPI_RESIDUAL,
                  nullptr, 1, n_dev, s)));
     PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln2_g, W + o.ln2_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
-    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, W + o.b1, e->Hm, rows_cap, Mlp, D, EPI_GELU, nullptr, 1,
+    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, e->c_Hm, W + o.b1, e->Hm, rows_cap, Mlp, D, EPI_GELU, nullptr, 1,
                  n_dev, s)));
-    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, W + o.b2, e->X[cur], rows_cap, D, Mlp, EPI_RESIDUAL,
+    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, e->c_X[cur], W + o.b2, e->X[cur], rows_cap, D, Mlp, EPI_RESIDUAL,
                  nullptr, 1, n_dev, s)));
   }
   const int* n_dev = e->fl[lst].n;
@@ -522,7 +523,7 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
       return cudaGetLastError() == cudaSuccess ? ET_OK : ET_ERR_CUDA;
     };
     if ((st = convert(e->off_patch_w, P, (int)D, e->Kp, &e->patch_w_t)) != ET_OK) return bail(st);
-    if (!make_tma_2d_bf16(&e->d_patch_w, e->patch_w_t, D, e->Kp, gemm_bf16_pick_bn((int)D), &err)) return bail(fail(e, ET_ERR_CUDA, err));
+    if (!make_tma_2d_bf16(&e->d_patch_w, e->patch_w_t, D, e->Kp, gemm_bf16_w_box_rows((int)D), &err)) return bail(fail(e, ET_ERR_CUDA, err));
     e->lb.resize(config->num_layers);
     for (int i = 0; i < config->num_layers; ++i) {
       LayerBf16& b = e->lb[i];
@@ -531,14 +532,16 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
       if ((st = convert(o.wo, (int)D, (int)D, (int)D, &b.wo_t)) != ET_OK) return bail(st);
       if ((st = convert(o.w1, (int)D, (int)M, (int)D, &b.w1_t)) != ET_OK) return bail(st);
       if ((st = convert(o.w2, (int)M, (int)D, (int)M, &b.w2_t)) != ET_OK) return bail(st);
-      bool ok = make_tma_2d_bf16(&b.d_wqkv, b.wqkv_t, 3 * D, D, gemm_bf16_pick_bn((int)(3 * D)), &err) &&
-                make_tma_2d_bf16(&b.d_wo, b.wo_t, D, D, gemm_bf16_pick_bn((int)D), &err) &&
-                make_tma_2d_bf16(&b.d_w1, b.w1_t, M, D, gemm_bf16_pick_bn((int)M), &err) &&
-                make_tma_2d_bf16(&b.d_w2, b.w2_t, D, M, gemm_bf16_pick_bn((int)D), &err);
+      bool ok = make_tma_2d_bf16(&b.d_wqkv, b.wqkv_t, 3 * D, D, gemm_bf16_w_box_rows((int)(3 * D)), &err) &&
+                make_tma_2d_bf16(&b.d_wo, b.wo_t, D, D, gemm_bf16_w_box_rows((int)D), &err) &&
+                make_tma_2d_bf16(&b.d_w1, b.w1_t, M, D, gemm_bf16_w_box_rows((int)M), &err) &&
+                make_tma_2d_bf16(&b.d_w2, b.w2_t, D, M, gemm_bf16_w_box_rows((int)D), &err);
       if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
     }
     bool ok = make_tma_2d_bf16(&e->d_Pm, e->Pm, rows, e->Kp, 128, &err) && make_tma_2d_bf16(&e->d_Xn, e->Xn, rows, D, 128, &err) &&
-              make_tma_2d_bf16(&e->d_O, e->O, rows, D, 128, &err) && make_tma_2d_bf16(&e->d_Hm, e->Hm, rows, M, 128, &err);
+              make_tma_2d_bf16(&e->d_O, e->O, rows, D, 128, &err) && make_tma_2d_bf16(&e->d_Hm, e->Hm, rows, M, 128, &err) &&
+              make_tma_out(&e->c_X[0], e->X[0], rows, D, true, &err) && make_tma_out(&e->c_X[1], e->X[1], rows, D, true, &err) &&
+              make_tma_out(&e->c_QKV, e->QKV, rows, 3 * D, false, &err) && make_tma_out(&e->c_Hm, e->Hm, rows, M, false, &err);
     if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
   }
   if (cudaDeviceSynchronize() != cudaSuccess) return bail(ET_ERR_CUDA);
@@ -731,11 +734,12 @@ et_status et_linear_bf16(const void* a_dev, const void* w_dev, const float* bias
   if (!a_dev || !w_dev || !bias_dev || !c_dev) return ET_ERR_INVALID_ARG;
   if (M < 1 || N < 8 || N % 8 != 0 || K < 8 || K % 8 != 0) return ET_ERR_SHAPE;
   if (epilogue < 0 || epilogue > 3 || (epilogue == 3 && (!table_dev || table_rows < 1))) return ET_ERR_INVALID_ARG;
-  TmaDesc da, dw;
+  TmaDesc da, dw, dc;
   const char* err = nullptr;
-  if (!make_tma_2d_bf16(&da, a_dev, M, K, 128, &err) || !make_tma_2d_bf16(&dw, w_dev, N, K, gemm_bf16_pick_bn(N), &err))
+  if (!make_tma_2d_bf16(&da, a_dev, M, K, 128, &err) || !make_tma_2d_bf16(&dw, w_dev, N, K, gemm_bf16_w_box_rows(N), &err) ||
+      !make_tma_out(&dc, c_dev, M, N, epilogue >= 2, &err))
     return ET_ERR_CUDA;
-  ET_CUDA0(launch_gemm_bf16(da, dw, bias_dev, c_dev, M, N, K, epilogue, gelu_tanh, table_dev, table_rows, nullptr, 1,
+  ET_CUDA0(launch_gemm_bf16(da, dw, dc, bias_dev, c_dev, M, N, K, epilogue, gelu_tanh, table_dev, table_rows, nullptr, 1,
                             status_dev, (cudaStream_t)cuda_stream));
   return ET_OK;
 }
