@@ -1,0 +1,420 @@
+// Per-frame multi-head attention on the 5th-generation tensor cores (tcgen05, accumulators in TMEM).
+//
+// One CTA owns 256 queries of one (frame, head) and sweeps the frame's keys in tiles of 128:
+//   warps 0..3  softmax group 0 (queries 0..127 of the CTA), warps 4..7 softmax group 1 (128..255):
+//               thread = query row = TMEM lane; reads the 128 logits of a tile row into registers with
+//               tcgen05.ld, keeps the running maximum and sum, writes P = exp2(S - m) as packed bf16 over
+//               the first half of the S columns with tcgen05.st.  While one group is in its softmax the
+//               tensor pipe works for the other.
+//   warp 8      TMA producer: Q (2 x 128 rows) once, then a ring of K / V tiles
+//   warp 9      allocates TMEM and issues all MMAs:  S = Q K^T  (SS form, 128 x 128 x 16 per instruction)
+//               and  O += P V  (TS form: P is read from TMEM, V from shared memory, MN-major)
+//   The control warpgroup (8..11) hands most of its registers to the softmax warpgroups (setmaxnreg).
+// The running maximum is only raised when the tile maximum exceeds it by more than 8 (in the log2
+// domain), so the rescale of O in TMEM is rare; P stays below 2^8, which bf16 represents without loss
+// of relative precision.  The final division by the row sum makes the result independent of that choice.
+//
+// Head dim 64 or 72.  A head row is 64 elements (one 128-byte swizzled row) plus, for 72, a tail of 8
+// elements kept as a separate 16-byte-per-row tile; the tail's contraction step pairs it with a block
+// of zeros so that K = 16 for the MMA.  Global memory keeps the packed [tokens][3*D] layout.
+#include "common.cuh"
+#include "tcgen05.cuh"
+
+namespace et {
+
+namespace {
+
+using namespace tc;
+
+constexpr int QT = 128;                 // queries per softmax group
+constexpr int QB = 2 * QT;              // queries per CTA
+constexpr int KT = 128;                 // keys per tile
+constexpr int KV_STAGES = 3;
+constexpr int MAIN_BYTES = 128 * 128;   // 128 rows x 64 bf16, 128-byte swizzle
+constexpr int TAIL_BYTES = 128 * 16;    // 128 rows x 8 bf16, rows 16 bytes apart
+constexpr int ATT_THREADS = 384;         // warps 0..7 softmax, 8 TMA, 9 MMA, 10..11 idle (complete the third warpgroup)
+constexpr int SOFTMAX_REGS = 200, CONTROL_REGS = 80;   // per-thread register budgets after setmaxnreg
+// setmaxnreg.inc blocks until the registers exist: the budgets must fit into what the CTA was launched with,
+// which is at least LAUNCH_REGS per thread (the kernel is compiled for exactly one CTA of ATT_THREADS per SM).
+constexpr int LAUNCH_REGS = 160;
+static_assert(SOFTMAX_REGS * 256 + CONTROL_REGS * 128 <= LAUNCH_REGS * ATT_THREADS, "register budgets exceed the CTA's allocation");
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+constexpr float RESCALE_GAP = 8.f;      // raise the running maximum only when a tile exceeds it by this (log2 domain)
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr int OFF_Q_MAIN = 0;
+constexpr int OFF_K_MAIN = OFF_Q_MAIN + 2 * MAIN_BYTES;
+constexpr int OFF_V_MAIN = OFF_K_MAIN + KV_STAGES * MAIN_BYTES;
+constexpr int OFF_Q_TAIL = OFF_V_MAIN + KV_STAGES * MAIN_BYTES;
+constexpr int OFF_K_TAIL = OFF_Q_TAIL + 2 * TAIL_BYTES;
+constexpr int OFF_V_TAIL = OFF_K_TAIL + KV_STAGES * TAIL_BYTES;
+constexpr int OFF_ZERO = OFF_V_TAIL + KV_STAGES * TAIL_BYTES;   // 2 KB of zeros: the second half of every tail step
+constexpr int OFF_BARS = OFF_ZERO + TAIL_BYTES;
+constexpr int ATT_SMEM_BYTES = OFF_BARS + 256 + 1024;
+
+// barrier slots
+constexpr int B_Q_FULL = 0, B_K_FULL = 1, B_V_FULL = B_K_FULL + KV_STAGES, B_KV_EMPTY = B_V_FULL + KV_STAGES,
+              B_S_FULL = B_KV_EMPTY + KV_STAGES, B_P_FULL = B_S_FULL + 2, B_O_READY = B_P_FULL + 2, B_COUNT = B_O_READY + 2;
+static_assert(B_COUNT * 8 + 8 <= 256, "barrier area");
+
+// TMEM columns: S of group t at t*128 (P aliases its first 64 columns), O of group t at 256 + t*80
+constexpr int TMEM_COLS = 512;
+constexpr int COL_O = 256, O_STRIDE = 80;
+
+struct AttnArgs {
+  bf16* out;
+  float* lse;
+  int n_cap, L, heads;
+  const int* n_frames_dev;
+  int* status;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// maximum of the (valid) logits of one 32-column chunk whose first column is c0
+template <bool MASK>
+__device__ __forceinline__ float row_max(const uint32_t (&r)[32], int c0, int nk) {
+  float a[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+  for (int i = 0; i < 32; ++i)
+    if (!MASK || c0 + i < nk) a[i & 3] = fmaxf(a[i & 3], __uint_as_float(r[i]));
+  return fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
+}
+
+// one 32-column chunk: p = 2^(s * scale - m) (0 beyond the frame's keys), row sums in four partial
+// accumulators, packed bf16 pairs to 16 TMEM columns at p_addr
+template <bool MASK>
+__device__ __forceinline__ void probs(const uint32_t (&r)[32], int c0, int nk, float scale2, float m, float (&ls)[4],
+                                      uint32_t p_addr) {
+  uint32_t pk[16];
+#pragma unroll
+  for (int i = 0; i < 32; i += 2) {
+    float p0 = ex2(fmaf(__uint_as_float(r[i]), scale2, -m));
+    float p1 = ex2(fmaf(__uint_as_float(r[i + 1]), scale2, -m));
+    if (MASK) {
+      if (c0 + i >= nk) p0 = 0.f;
+      if (c0 + i + 1 >= nk) p1 = 0.f;
+    }
+    ls[(i >> 1) & 1] += p0;
+    ls[2 + ((i >> 1) & 1)] += p1;
+    pk[i >> 1] = pack_bf16(p0, p1);
+  }
+  tmem_st16(p_addr, pk);
+}
+
+template <int DH>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_constant__ CUtensorMap tma_tail, AttnArgs g) {
+  constexpr bool HAS_TAIL = DH > 64;
+  static_assert(DH == 64 || DH == 72, "head dim");
+  const int n = g.n_frames_dev ? min(*g.n_frames_dev, g.n_cap) : g.n_cap;
+  const int f = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * QB;
+  if (f >= n) return;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* const gen_base = smem_raw + (base - raw);
+  const uint32_t bar_base = base + OFF_BARS;
+  auto bar = [&](int i) { return bar_base + 8u * (uint32_t)i; };
+  volatile uint32_t* tmem_ptr_slot = reinterpret_cast<volatile uint32_t*>(gen_base + OFF_BARS + 8 * B_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + OFF_BARS + 8 * B_COUNT + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int L = g.L, D = g.heads * DH;
+  const int n_tiles = (L + KT - 1) / KT;
+  const int row_base = f * L;
+
+  if (threadIdx.x == 0) {
+    mbar_init(bar(B_Q_FULL), 1);
+    for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar(B_K_FULL + s), 1); mbar_init(bar(B_V_FULL + s), 1); mbar_init(bar(B_KV_EMPTY + s), 1); }
+    for (int t = 0; t < 2; ++t) { mbar_init(bar(B_S_FULL + t), 1); mbar_init(bar(B_P_FULL + t), 4); mbar_init(bar(B_O_READY + t), 1); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = threadIdx.x; i < TAIL_BYTES / 16; i += ATT_THREADS)
+    reinterpret_cast<uint4*>(gen_base + OFF_ZERO)[i] = make_uint4(0u, 0u, 0u, 0u);
+  fence_async_smem();                   // the zeros are read by the tensor core (async proxy)
+  if (warp == 9) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32((const void*)tmem_ptr_slot)), "r"((uint32_t)TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  fence_before();
+  __syncthreads();
+  fence_after();
+  const uint32_t tmem_base = *tmem_ptr_slot;
+
+  auto keys_rounded = [&](int j) { return (min(KT, L - j * KT) + 15) & ~15; };   // MMA N / K extent of key tile j
+
+  if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(CONTROL_REGS));
+  if (warp == 8) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_main) : "memory");
+      if (HAS_TAIL) asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_tail) : "memory");
+      constexpr uint32_t TILE_TX = MAIN_BYTES + (HAS_TAIL ? TAIL_BYTES : 0);
+      mbar_arrive_expect_tx(bar(B_Q_FULL), 2 * TILE_TX);
+      for (int t = 0; t < 2; ++t) {
+        tma_load_2d(base + OFF_Q_MAIN + t * MAIN_BYTES, &tma_main, bar(B_Q_FULL), h * DH, row_base + q0 + t * QT);
+        if (HAS_TAIL) tma_load_2d(base + OFF_Q_TAIL + t * TAIL_BYTES, &tma_tail, bar(B_Q_FULL), h * DH + 64, row_base + q0 + t * QT);
+      }
+      for (int j = 0; j < n_tiles; ++j) {
+        const int s = j % KV_STAGES;
+        const uint32_t ph = (uint32_t)(j / KV_STAGES) & 1u;
+        if (!mbar_wait(bar(B_KV_EMPTY + s), ph ^ 1u, abort_flag)) break;
+        const int y = row_base + j * KT;
+        mbar_arrive_expect_tx(bar(B_K_FULL + s), TILE_TX);
+        tma_load_2d(base + OFF_K_MAIN + s * MAIN_BYTES, &tma_main, bar(B_K_FULL + s), D + h * DH, y);
+        if (HAS_TAIL) tma_load_2d(base + OFF_K_TAIL + s * TAIL_BYTES, &tma_tail, bar(B_K_FULL + s), D + h * DH + 64, y);
+        mbar_arrive_expect_tx(bar(B_V_FULL + s), TILE_TX);
+        tma_load_2d(base + OFF_V_MAIN + s * MAIN_BYTES, &tma_main, bar(B_V_FULL + s), 2 * D + h * DH, y);
+        if (HAS_TAIL) tma_load_2d(base + OFF_V_TAIL + s * TAIL_BYTES, &tma_tail, bar(B_V_FULL + s), 2 * D + h * DH + 64, y);
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    // The whole warp runs the loop (so that descriptors and addresses stay warp-uniform); one elected
+    // lane issues the MMAs and the commits.
+    {
+      constexpr uint32_t IDESC_PV_MAIN = idesc_bf16(128, 64, false, true), IDESC_PV_TAIL = idesc_bf16(128, 16, false, true);
+      // Descriptors of stage / group 0; the others differ by a multiple of the tile size in the address
+      // field (16-byte units, bits 0..13) and, for the tails, in the offset to the zero block (leading
+      // byte offset at bit 16 for the K-major Q / K tails, stride byte offset at bit 32 for the MN-major V tail).
+      const uint32_t zero = base + OFF_ZERO;
+      const uint64_t q_main0 = smem_desc(base + OFF_Q_MAIN, 16, 1024, 2), k_main0 = smem_desc(base + OFF_K_MAIN, 16, 1024, 2),
+                     v_main0 = smem_desc(base + OFF_V_MAIN, 16, 1024, 2);
+      const uint64_t q_tail0 = smem_desc(base + OFF_Q_TAIL, zero - (base + OFF_Q_TAIL), 128, 0),
+                     k_tail0 = smem_desc(base + OFF_K_TAIL, zero - (base + OFF_K_TAIL), 128, 0),
+                     v_tail0 = smem_desc(base + OFF_V_TAIL, 128, zero - (base + OFF_V_TAIL), 0);
+      constexpr uint64_t MAIN_STEP = MAIN_BYTES >> 4, TAIL_STEP = TAIL_BYTES >> 4;
+      auto main_desc = [&](uint64_t d0, int i) { return d0 + (uint64_t)i * MAIN_STEP; };
+      auto tail_desc = [&](uint64_t d0, int i, int off_shift) { return d0 + (uint64_t)i * TAIL_STEP - (((uint64_t)i * TAIL_STEP) << off_shift); };
+      bool ok = mbar_wait_warp(bar(B_Q_FULL), 0, abort_flag);
+      // step j issues  O += P V  of key tile j-1 and  S = Q K^T  of key tile j, group 0 then group 1
+      for (int j = 0; j <= n_tiles && ok; ++j) {
+        const int s = j % KV_STAGES;
+        if (j < n_tiles && !mbar_wait_warp(bar(B_K_FULL + s), (uint32_t)(j / KV_STAGES) & 1u, abort_flag)) { ok = false; break; }
+        for (int t = 0; t < 2 && ok; ++t) {
+          if (j > 0) {
+            const int jj = j - 1, sp = jj % KV_STAGES;
+            if (t == 0 && !mbar_wait_warp(bar(B_V_FULL + sp), (uint32_t)(jj / KV_STAGES) & 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_warp(bar(B_P_FULL + t), (uint32_t)jj & 1u, abort_flag)) { ok = false; break; }
+            fence_after();
+            const int ksteps = keys_rounded(jj) / 16;
+            const uint32_t o_col = tmem_base + COL_O + t * O_STRIDE;
+            uint32_t a = tmem_base + t * 128;                   // 16 keys = 8 columns of packed bf16 pairs
+            // V main part, MN-major with 128-byte swizzle: 16 keys = two 8-row groups of 1024 bytes.
+            // V tail, MN-major without swizzle: 8-key groups 128 bytes apart, second 8 columns = the zero block.
+            uint64_t dm = main_desc(v_main0, sp), dt = tail_desc(v_tail0, sp, 32);
+#pragma unroll 1
+            for (int ks = 0; ks < ksteps; ++ks) {
+              const uint32_t acc = (jj | ks) != 0 ? 1u : 0u;
+              mma_ts_elect(o_col, a, dm, IDESC_PV_MAIN, acc);
+              if (HAS_TAIL) mma_ts_elect(o_col + 64, a, dt, IDESC_PV_TAIL, acc);
+              a += 8; dm += 2048 >> 4; dt += 256 >> 4;          // the address field counts 16-byte units
+            }
+            commit_elect(bar(B_O_READY + t));
+            if (t == 1) commit_elect(bar(B_KV_EMPTY + sp));            // K and V of tile j-1 are no longer needed
+          }
+          if (j < n_tiles) {
+            const uint32_t idesc = idesc_bf16(128, keys_rounded(j), false, false);
+            const uint64_t qd = main_desc(q_main0, t), kd = main_desc(k_main0, s);
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)                       // 16 elements = 32 bytes inside the swizzle row
+              mma_ss_elect(tmem_base + t * 128, qd + 2 * ks, kd + 2 * ks, idesc, ks != 0 ? 1u : 0u);
+            // elements 64..71 and a block of zeros: two 8-element column blocks, the second one `lbo` bytes away
+            if (HAS_TAIL) mma_ss_elect(tmem_base + t * 128, tail_desc(q_tail0, t, 16), tail_desc(k_tail0, s, 16), idesc, 1u);
+            commit_elect(bar(B_S_FULL + t));
+          }
+        }
+      }
+    }
+  }
+  } else {
+    // ------------------------------------------------------------------ softmax groups
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(SOFTMAX_REGS));
+    const int t = warp >> 2;
+    const int quarter = warp & 3;                     // TMEM lanes 32*quarter .. +31
+    const int row = quarter * 32 + lane;
+    const int q = q0 + t * QT + row;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t s_addr = lane_addr + t * 128, o_addr = lane_addr + COL_O + t * O_STRIDE;
+    const float scale2 = LOG2E / sqrtf((float)DH);    // logits are kept in the log2 domain
+    float m = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      const int nk = min(KT, L - j * KT);
+      const int nch = (nk + 31) >> 5;
+      if (!mbar_wait_warp(bar(B_S_FULL + t), (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+      fence_after();
+      // the whole tile row (up to 128 logits) goes to registers with one wait
+      uint32_t r0[32], r1[32], r2[32], r3[32];
+      tmem_ld32_async(s_addr, r0);
+      if (nch > 1) tmem_ld32_async(s_addr + 32, r1);
+      if (nch > 2) tmem_ld32_async(s_addr + 64, r2);
+      if (nch > 3) tmem_ld32_async(s_addr + 96, r3);
+      tmem_wait_ld();
+      const bool full = nk == KT;
+      float mx;
+      if (full) {
+        mx = fmaxf(fmaxf(row_max<false>(r0, 0, nk), row_max<false>(r1, 32, nk)), fmaxf(row_max<false>(r2, 64, nk), row_max<false>(r3, 96, nk)));
+      } else {
+        mx = row_max<true>(r0, 0, nk);
+        if (nch > 1) mx = fmaxf(mx, row_max<true>(r1, 32, nk));
+        if (nch > 2) mx = fmaxf(mx, row_max<true>(r2, 64, nk));
+        if (nch > 3) mx = fmaxf(mx, row_max<true>(r3, 96, nk));
+      }
+      mx *= scale2;
+      if (__any_sync(0xffffffffu, mx > m + RESCALE_GAP)) {
+        const float m_new = fmaxf(m, mx);
+        if (j > 0) {
+          const float corr = ex2(m - m_new);
+          if (!mbar_wait_warp(bar(B_O_READY + t), (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
+          fence_after();
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+            uint32_t r[32];
+            tmem_ld32(o_addr + c * 32, r);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+            tmem_st32(o_addr + c * 32, r);
+          }
+          if (HAS_TAIL) {
+            uint32_t r[16];
+            tmem_ld16(o_addr + 64, r);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+            tmem_st16(o_addr + 64, r);
+          }
+          l *= corr;
+        }
+        m = m_new;
+      }
+      // P = exp2(S * scale - m) as packed bf16 over the first half of the S columns
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      if (full) {
+        probs<false>(r0, 0, nk, scale2, m, ls, s_addr);
+        probs<false>(r1, 32, nk, scale2, m, ls, s_addr + 16);
+        probs<false>(r2, 64, nk, scale2, m, ls, s_addr + 32);
+        probs<false>(r3, 96, nk, scale2, m, ls, s_addr + 48);
+      } else {
+        probs<true>(r0, 0, nk, scale2, m, ls, s_addr);
+        if (nch > 1) probs<true>(r1, 32, nk, scale2, m, ls, s_addr + 16);
+        if (nch > 2) probs<true>(r2, 64, nk, scale2, m, ls, s_addr + 32);
+        if (nch > 3) probs<true>(r3, 96, nk, scale2, m, ls, s_addr + 48);
+      }
+      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      tmem_wait_st();
+      fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(B_P_FULL + t));
+    }
+    if (ok && mbar_wait_warp(bar(B_O_READY + t), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
+      fence_after();
+      const float inv = 1.f / l;
+      bf16* orow = g.out + ((size_t)row_base + q) * D + (size_t)h * DH;
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        uint32_t r[32];
+        tmem_ld32(o_addr + c * 32, r);
+        if (q < L) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 o;
+            o.x = pack_bf16(__uint_as_float(r[i + 0]) * inv, __uint_as_float(r[i + 1]) * inv);
+            o.y = pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+            o.z = pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+            o.w = pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + c * 32 + i) = o;
+          }
+        }
+      }
+      if (HAS_TAIL) {
+        uint32_t r[8];
+        tmem_ld8(o_addr + 64, r);
+        if (q < L) {
+          uint4 o;
+          o.x = pack_bf16(__uint_as_float(r[0]) * inv, __uint_as_float(r[1]) * inv);
+          o.y = pack_bf16(__uint_as_float(r[2]) * inv, __uint_as_float(r[3]) * inv);
+          o.z = pack_bf16(__uint_as_float(r[4]) * inv, __uint_as_float(r[5]) * inv);
+          o.w = pack_bf16(__uint_as_float(r[6]) * inv, __uint_as_float(r[7]) * inv);
+          *reinterpret_cast<uint4*>(orow + 64) = o;
+        }
+      }
+      if (q < L) g.lse[((size_t)f * g.heads + h) * L + q] = (m + log2f(l)) * LN2;
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  __syncwarp();
+  fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) __nanosleep(1000);      // let copies in flight land
+    if (threadIdx.x == 0 && g.status) atomicExch(g.status, (int)DS_WAIT_EXPIRED);
+    __syncthreads();
+  }
+  if (warp == 9) {
+    fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+  }
+}
+
+bool encode_map(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_cols, CUtensorMapSwizzle sw) {
+  EncodeTiledFn fn = tensor_map_encoder();
+  if (!fn) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) || ((cols * 2) & 15u)) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * 2};
+  const cuuint32_t box[2] = {box_cols, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(reinterpret_cast<CUtensorMap*>(out->bytes), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int DH>
+cudaError_t run(const AttnMaps& maps, const AttnArgs& a, cudaStream_t s) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  ET_COUNT_LAUNCH();
+  attention_tc_kernel<DH><<<dim3(cdiv(a.L, QB), a.heads, a.n_cap), ATT_THREADS, ATT_SMEM_BYTES, s>>>(
+      *reinterpret_cast<const CUtensorMap*>(maps.main.bytes), *reinterpret_cast<const CUtensorMap*>(maps.tail.bytes), a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool attention_tc_supported(int dh) { return dh == 64 || dh == 72; }
+
+bool make_attention_maps(AttnMaps* out, const bf16* qkv, long long rows, int heads, int dh) {
+  if (!attention_tc_supported(dh)) return false;
+  const uint64_t cols = (uint64_t)3 * heads * dh;
+  if (!encode_map(&out->main, qkv, (uint64_t)rows, cols, 64, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
+  if (dh > 64 && !encode_map(&out->tail, qkv, (uint64_t)rows, cols, 8, CU_TENSOR_MAP_SWIZZLE_NONE)) return false;
+  if (dh <= 64) out->tail = out->main;
+  return true;
+}
+
+cudaError_t launch_attention_tc(const AttnMaps& maps, bf16* out, float* lse, int n_cap, int L, int heads, int dh,
+                                const int* n_frames_dev, int* status_dev, cudaStream_t s) {
+  if (n_cap <= 0) return cudaSuccess;
+  AttnArgs a{out, lse, n_cap, L, heads, n_frames_dev, status_dev};
+  if (dh == 72) return run<72>(maps, a, s);
+  if (dh == 64) return run<64>(maps, a, s);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace et

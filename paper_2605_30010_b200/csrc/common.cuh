@@ -90,6 +90,12 @@ void launch_attention_f32(const float* qkv, float* out, float* lse, int n_cap, i
 void launch_attention_bf16(const bf16* qkv, bf16* out, float* lse, int n_cap, int L, int heads, int dh,
                            const int* n_frames_dev, cudaStream_t s);
 bool attention_bf16_supported(int L, int heads, int dh);
+// tcgen05 attention (attention_tcgen05.cu): head dims 64 and 72.  The maps describe qkv [rows][3*D] bf16.
+struct AttnMaps { TmaDesc main, tail; };
+bool attention_tc_supported(int dh);
+bool make_attention_maps(AttnMaps* out, const bf16* qkv, long long rows, int heads, int dh);
+cudaError_t launch_attention_tc(const AttnMaps& maps, bf16* out, float* lse, int n_cap, int L, int heads, int dh,
+                                const int* n_frames_dev, int* status_dev, cudaStream_t s);
 // partial[f][h][j] = sum_q exp(s(q,j) - lse[f][h][q]);  score[f][j] = sum_h partial / (heads*L)
 void launch_attention_scores_f32(const float* qkv, const float* lse, float* partial, float* score, int n_cap, int L,
                                  int heads, int dh, const int* n_frames_dev, cudaStream_t s);

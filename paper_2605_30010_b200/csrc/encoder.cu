@@ -67,6 +67,8 @@ struct et_encoder {
   void *Pm = nullptr, *Xn = nullptr, *QKV = nullptr, *O = nullptr, *Hm = nullptr;
   TmaDesc d_Pm, d_Xn, d_O, d_Hm;                   // operand (A) maps
   TmaDesc c_X[2], c_QKV, c_Hm;                      // output (C) maps
+  AttnMaps attn_maps;                               // QKV as seen by the tcgen05 attention kernel
+  bool attn_tc = false;
   float *lse = nullptr, *score_partial = nullptr, *scores = nullptr, *cosbuf = nullptr, *simbuf = nullptr;
   float* frames_stage = nullptr;               // device staging for the *_host entry point (lazy)
 
@@ -299,7 +301,8 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.wqkv, b ? b->d_wqkv : none, e->c_QKV, W + o.bqkv, e->QKV, rows_cap, 3 * D, D, EPI_STORE,
                  nullptr, 1, n_dev, s)));
     PROF(ET_CAT_ATTENTION, {
-      if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, s);
+      if (e->attn_tc) ET_CUDA(e, launch_attention_tc(e->attn_maps, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, e->d_small + 10, s));
+      else if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, s);
       else launch_attention_f32((const float*)e->QKV, (float*)e->O, e->lse, T, L, H, dh, n_dev, s);
     });
     if (layer == c.num_layers - 1) {
@@ -543,6 +546,11 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
               make_tma_out(&e->c_X[0], e->X[0], rows, D, true, &err) && make_tma_out(&e->c_X[1], e->X[1], rows, D, true, &err) &&
               make_tma_out(&e->c_QKV, e->QKV, rows, 3 * D, false, &err) && make_tma_out(&e->c_Hm, e->Hm, rows, M, false, &err);
     if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
+    if (attention_tc_supported(e->dh)) {
+      if (!make_attention_maps(&e->attn_maps, (const bf16*)e->QKV, (long long)rows, config->heads, e->dh))
+        return bail(fail(e, ET_ERR_CUDA, "tensor map of the attention operands"));
+      e->attn_tc = true;
+    }
   }
   if (cudaDeviceSynchronize() != cudaSuccess) return bail(ET_ERR_CUDA);
   *out = e;
@@ -751,6 +759,12 @@ et_status et_attention(const void* qkv_dev, void* out_dev, float* lse_dev, int n
   cudaStream_t s = (cudaStream_t)cuda_stream;
   if (dtype == ET_BF16) {
     if (head_dim % 8 != 0) return ET_ERR_SHAPE;
+    if (attention_tc_supported(head_dim)) {
+      AttnMaps maps;
+      if (!make_attention_maps(&maps, (const bf16*)qkv_dev, (long long)n * L, heads, head_dim)) return ET_ERR_CUDA;
+      ET_CUDA0(launch_attention_tc(maps, (bf16*)out_dev, lse_dev, n, L, heads, head_dim, nullptr, nullptr, s));
+      return ET_OK;
+    }
     launch_attention_bf16((const bf16*)qkv_dev, (bf16*)out_dev, lse_dev, n, L, heads, head_dim, nullptr, s);
   } else if (dtype == ET_F32) {
     launch_attention_f32((const float*)qkv_dev, (float*)out_dev, lse_dev, n, L, heads, head_dim, nullptr, s);
