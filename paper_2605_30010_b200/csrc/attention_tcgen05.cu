@@ -1,6 +1,7 @@
 // Per-frame multi-head attention on the 5th-generation tensor cores (tcgen05, accumulators in TMEM).
 //
-// One CTA owns 256 queries of one (frame, head) and sweeps the frame's keys in tiles of 128:
+// Persistent kernel, one CTA per SM.  A work item is 256 queries of one (frame, head); the CTA sweeps the
+// frame's keys in tiles of 128 and goes on to its next item without draining its pipelines:
 //   warps 0..3  softmax group 0 (queries 0..127 of the CTA), warps 4..7 softmax group 1 (128..255):
 //               thread = query row = TMEM lane; reads the 128 logits of a tile row into registers with
 //               tcgen05.ld, keeps the running maximum and sum, writes P = exp2(S - m) as packed bf16 over
@@ -15,8 +16,9 @@
 // of relative precision.  The final division by the row sum makes the result independent of that choice.
 //
 // Head dim 64 or 72.  A head row is 64 elements (one 128-byte swizzled row) plus, for 72, a tail of 8
-// elements kept as a separate 16-byte-per-row tile; the tail's contraction step pairs it with a block
-// of zeros so that K = 16 for the MMA.  Global memory keeps the packed [tokens][3*D] layout.
+// elements: for Q and K a separate 16-byte-per-row tile whose contraction step pairs it with a block of
+// zeros (K = 16 for the MMA); for V a second swizzled 64-column box, so that O += P V is one MMA of N = 80
+// per 16 keys (its columns 72..79 are never read).  Global memory keeps the packed [tokens][3*D] layout.
 #include "common.cuh"
 #include "tcgen05.cuh"
 
@@ -45,17 +47,18 @@ constexpr float RESCALE_GAP = 8.f;      // raise the running maximum only when a
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr int OFF_Q_MAIN = 0;
 constexpr int OFF_K_MAIN = OFF_Q_MAIN + 2 * MAIN_BYTES;
+constexpr int V_STAGE_BYTES = 2 * MAIN_BYTES;                   // columns 0..63 of the head, then the 64 columns from 64 on
 constexpr int OFF_V_MAIN = OFF_K_MAIN + KV_STAGES * MAIN_BYTES;
-constexpr int OFF_Q_TAIL = OFF_V_MAIN + KV_STAGES * MAIN_BYTES;
+constexpr int OFF_Q_TAIL = OFF_V_MAIN + KV_STAGES * V_STAGE_BYTES;
 constexpr int OFF_K_TAIL = OFF_Q_TAIL + 2 * TAIL_BYTES;
-constexpr int OFF_V_TAIL = OFF_K_TAIL + KV_STAGES * TAIL_BYTES;
-constexpr int OFF_ZERO = OFF_V_TAIL + KV_STAGES * TAIL_BYTES;   // 2 KB of zeros: the second half of every tail step
+constexpr int OFF_ZERO = OFF_K_TAIL + KV_STAGES * TAIL_BYTES;   // 2 KB of zeros: the second half of the Q K^T tail step
 constexpr int OFF_BARS = OFF_ZERO + TAIL_BYTES;
 constexpr int ATT_SMEM_BYTES = OFF_BARS + 256 + 1024;
 
 // barrier slots
 constexpr int B_Q_FULL = 0, B_K_FULL = 1, B_V_FULL = B_K_FULL + KV_STAGES, B_KV_EMPTY = B_V_FULL + KV_STAGES,
-              B_S_FULL = B_KV_EMPTY + KV_STAGES, B_P_FULL = B_S_FULL + 2, B_O_READY = B_P_FULL + 2, B_COUNT = B_O_READY + 2;
+              B_S_FULL = B_KV_EMPTY + KV_STAGES, B_P_FULL = B_S_FULL + 2, B_O_READY = B_P_FULL + 2, B_Q_EMPTY = B_O_READY + 2,
+              B_COUNT = B_Q_EMPTY + 1;
 static_assert(B_COUNT * 8 + 8 <= 256, "barrier area");
 
 // TMEM columns: S of group t at t*128 (P aliases its first 64 columns), O of group t at 256 + t*80
@@ -113,8 +116,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
   constexpr bool HAS_TAIL = DH > 64;
   static_assert(DH == 64 || DH == 72, "head dim");
   const int n = g.n_frames_dev ? min(*g.n_frames_dev, g.n_cap) : g.n_cap;
-  const int f = blockIdx.z, h = blockIdx.y, q0 = blockIdx.x * QB;
-  if (f >= n) return;
+  const int L = g.L, D = g.heads * DH;
+  const int n_tiles = (L + KT - 1) / KT;
+  const int q_blocks = (L + QB - 1) / QB;
+  // Work items (frame, head, block of 256 queries), query block fastest: the CTAs that run side by side
+  // share the K / V of one (frame, head) in L2.  This CTA takes items blockIdx.x, + gridDim.x, ...
+  const int n_items = n * g.heads * q_blocks;
+  const int my_items = (int)blockIdx.x < n_items ? (n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+  if (my_items == 0) return;
+  const int total_tiles = my_items * n_tiles;          // key tiles this CTA sweeps, over all its items
+  auto item_coords = [&](int i, int& f, int& h, int& q0) {
+    const int item = (int)blockIdx.x + i * (int)gridDim.x;
+    q0 = (item % q_blocks) * QB;
+    h = (item / q_blocks) % g.heads;
+    f = item / (q_blocks * g.heads);
+  };
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -126,12 +142,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + OFF_BARS + 8 * B_COUNT + 4);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int L = g.L, D = g.heads * DH;
-  const int n_tiles = (L + KT - 1) / KT;
-  const int row_base = f * L;
 
   if (threadIdx.x == 0) {
     mbar_init(bar(B_Q_FULL), 1);
+    mbar_init(bar(B_Q_EMPTY), 1);
     for (int s = 0; s < KV_STAGES; ++s) { mbar_init(bar(B_K_FULL + s), 1); mbar_init(bar(B_V_FULL + s), 1); mbar_init(bar(B_KV_EMPTY + s), 1); }
     for (int t = 0; t < 2; ++t) { mbar_init(bar(B_S_FULL + t), 1); mbar_init(bar(B_P_FULL + t), 4); mbar_init(bar(B_O_READY + t), 1); }
     *abort_flag = 0;
@@ -150,7 +164,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
   fence_after();
   const uint32_t tmem_base = *tmem_ptr_slot;
 
-  auto keys_rounded = [&](int j) { return (min(KT, L - j * KT) + 15) & ~15; };   // MMA N / K extent of key tile j
+  auto keys_rounded = [&](int j) { return (min(KT, L - j * KT) + 15) & ~15; };   // MMA N / K extent of key tile j of an item
 
   if (warp >= 8) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(CONTROL_REGS));
@@ -160,22 +174,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_main) : "memory");
       if (HAS_TAIL) asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_tail) : "memory");
       constexpr uint32_t TILE_TX = MAIN_BYTES + (HAS_TAIL ? TAIL_BYTES : 0);
-      mbar_arrive_expect_tx(bar(B_Q_FULL), 2 * TILE_TX);
-      for (int t = 0; t < 2; ++t) {
-        tma_load_2d(base + OFF_Q_MAIN + t * MAIN_BYTES, &tma_main, bar(B_Q_FULL), h * DH, row_base + q0 + t * QT);
-        if (HAS_TAIL) tma_load_2d(base + OFF_Q_TAIL + t * TAIL_BYTES, &tma_tail, bar(B_Q_FULL), h * DH + 64, row_base + q0 + t * QT);
-      }
-      for (int j = 0; j < n_tiles; ++j) {
-        const int s = j % KV_STAGES;
-        const uint32_t ph = (uint32_t)(j / KV_STAGES) & 1u;
-        if (!mbar_wait(bar(B_KV_EMPTY + s), ph ^ 1u, abort_flag)) break;
-        const int y = row_base + j * KT;
-        mbar_arrive_expect_tx(bar(B_K_FULL + s), TILE_TX);
-        tma_load_2d(base + OFF_K_MAIN + s * MAIN_BYTES, &tma_main, bar(B_K_FULL + s), D + h * DH, y);
-        if (HAS_TAIL) tma_load_2d(base + OFF_K_TAIL + s * TAIL_BYTES, &tma_tail, bar(B_K_FULL + s), D + h * DH + 64, y);
-        mbar_arrive_expect_tx(bar(B_V_FULL + s), TILE_TX);
-        tma_load_2d(base + OFF_V_MAIN + s * MAIN_BYTES, &tma_main, bar(B_V_FULL + s), 2 * D + h * DH, y);
-        if (HAS_TAIL) tma_load_2d(base + OFF_V_TAIL + s * TAIL_BYTES, &tma_tail, bar(B_V_FULL + s), 2 * D + h * DH + 64, y);
+      bool ok = true;
+      int gt = 0;                                        // key tiles loaded so far: ring stage and phase
+      for (int i = 0; i < my_items && ok; ++i) {
+        int f, h, q0;
+        item_coords(i, f, h, q0);
+        const int row_base = f * L;
+        // Q of the previous item is free once its last Q K^T has completed
+        if (i > 0 && !mbar_wait(bar(B_Q_EMPTY), (uint32_t)(i - 1) & 1u, abort_flag)) break;
+        mbar_arrive_expect_tx(bar(B_Q_FULL), 2 * TILE_TX);
+        for (int t = 0; t < 2; ++t) {
+          tma_load_2d(base + OFF_Q_MAIN + t * MAIN_BYTES, &tma_main, bar(B_Q_FULL), h * DH, row_base + q0 + t * QT);
+          if (HAS_TAIL) tma_load_2d(base + OFF_Q_TAIL + t * TAIL_BYTES, &tma_tail, bar(B_Q_FULL), h * DH + 64, row_base + q0 + t * QT);
+        }
+        for (int j = 0; j < n_tiles; ++j, ++gt) {
+          const int s = gt % KV_STAGES;
+          const uint32_t ph = (uint32_t)(gt / KV_STAGES) & 1u;
+          if (!mbar_wait(bar(B_KV_EMPTY + s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          const int y = row_base + j * KT;
+          mbar_arrive_expect_tx(bar(B_K_FULL + s), TILE_TX);
+          tma_load_2d(base + OFF_K_MAIN + s * MAIN_BYTES, &tma_main, bar(B_K_FULL + s), D + h * DH, y);
+          if (HAS_TAIL) tma_load_2d(base + OFF_K_TAIL + s * TAIL_BYTES, &tma_tail, bar(B_K_FULL + s), D + h * DH + 64, y);
+          // V: a second 64-column box starting at column 64 of the head; only its first 8 columns belong to
+          // the head, the rest (the next head, or zeros past the row end) lands in output columns nobody reads
+          mbar_arrive_expect_tx(bar(B_V_FULL + s), HAS_TAIL ? V_STAGE_BYTES : MAIN_BYTES);
+          tma_load_2d(base + OFF_V_MAIN + s * V_STAGE_BYTES, &tma_main, bar(B_V_FULL + s), 2 * D + h * DH, y);
+          if (HAS_TAIL) tma_load_2d(base + OFF_V_MAIN + s * V_STAGE_BYTES + MAIN_BYTES, &tma_main, bar(B_V_FULL + s), 2 * D + h * DH + 64, y);
+        }
       }
     }
   } else if (warp == 9) {
@@ -183,47 +208,49 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
     // The whole warp runs the loop (so that descriptors and addresses stay warp-uniform); one elected
     // lane issues the MMAs and the commits.
     {
-      constexpr uint32_t IDESC_PV_MAIN = idesc_bf16(128, 64, false, true), IDESC_PV_TAIL = idesc_bf16(128, 16, false, true);
+      constexpr uint32_t IDESC_PV = idesc_bf16(128, HAS_TAIL ? 80 : 64, false, true);
       // Descriptors of stage / group 0; the others differ by a multiple of the tile size in the address
-      // field (16-byte units, bits 0..13) and, for the tails, in the offset to the zero block (leading
-      // byte offset at bit 16 for the K-major Q / K tails, stride byte offset at bit 32 for the MN-major V tail).
+      // field (16-byte units, bits 0..13) and, for the Q / K tails, in the offset to the zero block
+      // (leading byte offset at bit 16).  V is MN-major with 128-byte swizzle: 64 columns per atom, the
+      // second atom MAIN_BYTES further (leading byte offset), 8-key groups 1024 bytes apart.
       const uint32_t zero = base + OFF_ZERO;
       const uint64_t q_main0 = smem_desc(base + OFF_Q_MAIN, 16, 1024, 2), k_main0 = smem_desc(base + OFF_K_MAIN, 16, 1024, 2),
-                     v_main0 = smem_desc(base + OFF_V_MAIN, 16, 1024, 2);
+                     v_main0 = smem_desc(base + OFF_V_MAIN, MAIN_BYTES, 1024, 2);
       const uint64_t q_tail0 = smem_desc(base + OFF_Q_TAIL, zero - (base + OFF_Q_TAIL), 128, 0),
-                     k_tail0 = smem_desc(base + OFF_K_TAIL, zero - (base + OFF_K_TAIL), 128, 0),
-                     v_tail0 = smem_desc(base + OFF_V_TAIL, 128, zero - (base + OFF_V_TAIL), 0);
+                     k_tail0 = smem_desc(base + OFF_K_TAIL, zero - (base + OFF_K_TAIL), 128, 0);
       constexpr uint64_t MAIN_STEP = MAIN_BYTES >> 4, TAIL_STEP = TAIL_BYTES >> 4;
       auto main_desc = [&](uint64_t d0, int i) { return d0 + (uint64_t)i * MAIN_STEP; };
       auto tail_desc = [&](uint64_t d0, int i, int off_shift) { return d0 + (uint64_t)i * TAIL_STEP - (((uint64_t)i * TAIL_STEP) << off_shift); };
-      bool ok = mbar_wait_warp(bar(B_Q_FULL), 0, abort_flag);
-      // step j issues  O += P V  of key tile j-1 and  S = Q K^T  of key tile j, group 0 then group 1
-      for (int j = 0; j <= n_tiles && ok; ++j) {
-        const int s = j % KV_STAGES;
-        if (j < n_tiles && !mbar_wait_warp(bar(B_K_FULL + s), (uint32_t)(j / KV_STAGES) & 1u, abort_flag)) { ok = false; break; }
+      // Step g issues  O += P V  of key tile g-1 and  S = Q K^T  of key tile g (group 0, then group 1),
+      // g counting the key tiles of all items of this CTA: the first Q K^T of an item overlaps the last
+      // softmax of the item before it.
+      bool ok = true;
+      for (int gt = 0; gt <= total_tiles && ok; ++gt) {
+        const int s = gt % KV_STAGES, j = gt % n_tiles;
         for (int t = 0; t < 2 && ok; ++t) {
-          if (j > 0) {
-            const int jj = j - 1, sp = jj % KV_STAGES;
-            if (t == 0 && !mbar_wait_warp(bar(B_V_FULL + sp), (uint32_t)(jj / KV_STAGES) & 1u, abort_flag)) { ok = false; break; }
-            if (!mbar_wait_warp(bar(B_P_FULL + t), (uint32_t)jj & 1u, abort_flag)) { ok = false; break; }
+          if (gt > 0) {
+            const int gp = gt - 1, jj = gp % n_tiles, sp = gp % KV_STAGES;
+            if (t == 0 && !mbar_wait_warp(bar(B_V_FULL + sp), (uint32_t)(gp / KV_STAGES) & 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_warp(bar(B_P_FULL + t), (uint32_t)gp & 1u, abort_flag)) { ok = false; break; }
             fence_after();
             const int ksteps = keys_rounded(jj) / 16;
             const uint32_t o_col = tmem_base + COL_O + t * O_STRIDE;
             uint32_t a = tmem_base + t * 128;                   // 16 keys = 8 columns of packed bf16 pairs
-            // V main part, MN-major with 128-byte swizzle: 16 keys = two 8-row groups of 1024 bytes.
-            // V tail, MN-major without swizzle: 8-key groups 128 bytes apart, second 8 columns = the zero block.
-            uint64_t dm = main_desc(v_main0, sp), dt = tail_desc(v_tail0, sp, 32);
+            uint64_t dv = v_main0 + (uint64_t)sp * (V_STAGE_BYTES >> 4);
 #pragma unroll 1
             for (int ks = 0; ks < ksteps; ++ks) {
-              const uint32_t acc = (jj | ks) != 0 ? 1u : 0u;
-              mma_ts_elect(o_col, a, dm, IDESC_PV_MAIN, acc);
-              if (HAS_TAIL) mma_ts_elect(o_col + 64, a, dt, IDESC_PV_TAIL, acc);
-              a += 8; dm += 2048 >> 4; dt += 256 >> 4;          // the address field counts 16-byte units
+              mma_ts_elect(o_col, a, dv, IDESC_PV, (jj | ks) != 0 ? 1u : 0u);   // the first tile of an item overwrites O
+              a += 8; dv += 2048 >> 4;                           // 16 keys = two 8-row groups; 16-byte units
             }
             commit_elect(bar(B_O_READY + t));
-            if (t == 1) commit_elect(bar(B_KV_EMPTY + sp));            // K and V of tile j-1 are no longer needed
+            if (t == 1) commit_elect(bar(B_KV_EMPTY + sp));      // K and V of that tile are no longer needed
           }
-          if (j < n_tiles) {
+          if (gt < total_tiles) {
+            if (t == 0) {      // operands of this tile (waited for only now: the P V above must not wait for the next item's Q)
+              if (j == 0 && !mbar_wait_warp(bar(B_Q_FULL), (uint32_t)(gt / n_tiles) & 1u, abort_flag)) { ok = false; break; }
+              if (!mbar_wait_warp(bar(B_K_FULL + s), (uint32_t)(gt / KV_STAGES) & 1u, abort_flag)) { ok = false; break; }
+              fence_after();
+            }
             const uint32_t idesc = idesc_bf16(128, keys_rounded(j), false, false);
             const uint64_t qd = main_desc(q_main0, t), kd = main_desc(k_main0, s);
 #pragma unroll
@@ -232,6 +259,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
             // elements 64..71 and a block of zeros: two 8-element column blocks, the second one `lbo` bytes away
             if (HAS_TAIL) mma_ss_elect(tmem_base + t * 128, tail_desc(q_tail0, t, 16), tail_desc(k_tail0, s, 16), idesc, 1u);
             commit_elect(bar(B_S_FULL + t));
+            if (t == 1 && j == n_tiles - 1) commit_elect(bar(B_Q_EMPTY));   // the item's last read of Q
           }
         }
       }
@@ -243,16 +271,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
     const int t = warp >> 2;
     const int quarter = warp & 3;                     // TMEM lanes 32*quarter .. +31
     const int row = quarter * 32 + lane;
-    const int q = q0 + t * QT + row;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const uint32_t s_addr = lane_addr + t * 128, o_addr = lane_addr + COL_O + t * O_STRIDE;
     const float scale2 = LOG2E / sqrtf((float)DH);    // logits are kept in the log2 domain
-    float m = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
+    int gt = 0;                                       // key tiles processed so far (barrier phases)
+    for (int i = 0; i < my_items && ok; ++i) {
+    int f, h, q0;
+    item_coords(i, f, h, q0);
+    const int row_base = f * L, q = q0 + t * QT + row;
+    float m = -INFINITY, l = 0.f;
+    for (int j = 0; j < n_tiles; ++j, ++gt) {
       const int nk = min(KT, L - j * KT);
       const int nch = (nk + 31) >> 5;
-      if (!mbar_wait_warp(bar(B_S_FULL + t), (uint32_t)j & 1u, abort_flag)) { ok = false; break; }
+      if (!mbar_wait_warp(bar(B_S_FULL + t), (uint32_t)gt & 1u, abort_flag)) { ok = false; break; }
       fence_after();
       // the whole tile row (up to 128 logits) goes to registers with one wait
       uint32_t r0[32], r1[32], r2[32], r3[32];
@@ -276,7 +308,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
         const float m_new = fmaxf(m, mx);
         if (j > 0) {
           const float corr = ex2(m - m_new);
-          if (!mbar_wait_warp(bar(B_O_READY + t), (uint32_t)(j - 1) & 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait_warp(bar(B_O_READY + t), (uint32_t)(gt - 1) & 1u, abort_flag)) { ok = false; break; }
           fence_after();
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
@@ -316,7 +348,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(B_P_FULL + t));
     }
-    if (ok && mbar_wait_warp(bar(B_O_READY + t), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
+    if (!ok) break;
+    if (!mbar_wait_warp(bar(B_O_READY + t), (uint32_t)(gt - 1) & 1u, abort_flag)) { ok = false; break; }
+    {
       fence_after();
       const float inv = 1.f / l;
       bf16* orow = g.out + ((size_t)row_base + q) * D + (size_t)h * DH;
@@ -350,6 +384,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
       }
       if (q < L) g.lse[((size_t)f * g.heads + h) * L + q] = (m + log2f(l)) * LN2;
     }
+    }   // items
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -390,7 +425,15 @@ cudaError_t run(const AttnMaps& maps, const AttnArgs& a, cudaStream_t s) {
     configured = true;
   }
   ET_COUNT_LAUNCH();
-  attention_tc_kernel<DH><<<dim3(cdiv(a.L, QB), a.heads, a.n_cap), ATT_THREADS, ATT_SMEM_BYTES, s>>>(
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
+  const long long items_cap = (long long)cdiv(a.L, QB) * a.heads * a.n_cap;
+  const int grid = (int)(items_cap < sms ? items_cap : sms);      // one CTA per SM, each loops over its items
+  attention_tc_kernel<DH><<<grid, ATT_THREADS, ATT_SMEM_BYTES, s>>>(
       *reinterpret_cast<const CUtensorMap*>(maps.main.bytes), *reinterpret_cast<const CUtensorMap*>(maps.tail.bytes), a);
   return cudaGetLastError();
 }
