@@ -14,7 +14,7 @@ namespace et {
 constexpr int COS_RUN = 8;   // pairs per warp job
 
 template <int NV>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 token_cos_kernel(const float* __restrict__ x, float* __restrict__ cosbuf, int n_cap, int L, int D,
                  const int* __restrict__ n_frames_dev) {
   const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
@@ -29,30 +29,49 @@ token_cos_kernel(const float* __restrict__ x, float* __restrict__ cosbuf, int n_
     const int l = job % L, run = job / L;
     const int t0 = run * COS_RUN, t1 = min(t0 + COS_RUN, n_pairs);
     const float4* row = reinterpret_cast<const float4*>(x + (size_t)t0 * frame_stride + (size_t)l * D);
-    float4 prev[NV];
+    float4 prev[NV], cur[NV];
     float np = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
       const int i = lane + 32 * j;
       prev[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-      np += (prev[j].x * prev[j].x + prev[j].y * prev[j].y) + (prev[j].z * prev[j].z + prev[j].w * prev[j].w);
     }
+    row = reinterpret_cast<const float4*>(x + (size_t)(t0 + 1) * frame_stride + (size_t)l * D);
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const int i = lane + 32 * j;
+      cur[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int j = 0; j < NV; ++j)
+      np += (prev[j].x * prev[j].x + prev[j].y * prev[j].y) + (prev[j].z * prev[j].z + prev[j].w * prev[j].w);
     np = warp_sum(np);
     for (int t = t0; t < t1; ++t) {
-      row = reinterpret_cast<const float4*>(x + (size_t)(t + 1) * frame_stride + (size_t)l * D);
+      // the row after next is requested before this pair is reduced, so that loads stay in flight
+      float4 nxt[NV];
+      if (t + 1 < t1) {
+        row = reinterpret_cast<const float4*>(x + (size_t)(t + 2) * frame_stride + (size_t)l * D);
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+          const int i = lane + 32 * j;
+          nxt[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
       float dot = 0.f, nc = 0.f;
 #pragma unroll
       for (int j = 0; j < NV; ++j) {
-        const int i = lane + 32 * j;
-        const float4 c = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 c = cur[j];
         dot += (prev[j].x * c.x + prev[j].y * c.y) + (prev[j].z * c.z + prev[j].w * c.w);
         nc += (c.x * c.x + c.y * c.y) + (c.z * c.z + c.w * c.w);
-        prev[j] = c;
       }
       dot = warp_sum(dot);
       nc = warp_sum(nc);
       if (lane == 0) cosbuf[(size_t)t * L + l] = dot / fmaxf(sqrtf(np) * sqrtf(nc), 1e-8f);
       np = nc;
+      if (t + 1 < t1) {
+#pragma unroll
+        for (int j = 0; j < NV; ++j) { prev[j] = cur[j]; cur[j] = nxt[j]; }
+      }
     }
   }
 }
@@ -61,10 +80,10 @@ void launch_token_cosines(const float* x, float* cos_scratch, int n_cap, int L, 
                           cudaStream_t s) {
   if (n_cap < 2) return;
   const int runs = cdiv(n_cap - 1, COS_RUN);
-  const int blocks = min(cdiv((long long)runs * L, 8), 148 * 8);
+  const int blocks = min(cdiv((long long)runs * L, 4), 148 * 16);
   const int need = cdiv(D / 4, 32);
   ET_COUNT_LAUNCH();
-#define ET_COS(NV) token_cos_kernel<NV><<<blocks, 256, 0, s>>>(x, cos_scratch, n_cap, L, D, n_frames_dev)
+#define ET_COS(NV) token_cos_kernel<NV><<<blocks, 128, 0, s>>>(x, cos_scratch, n_cap, L, D, n_frames_dev)
   if (need <= 1) ET_COS(1);
   else if (need <= 2) ET_COS(2);
   else if (need <= 4) ET_COS(4);
