@@ -293,6 +293,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
       if (nch > 2) tmem_ld32_async(s_addr + 64, r2);
       if (nch > 3) tmem_ld32_async(s_addr + 96, r3);
       tmem_wait_ld();
+      tmem_regs_ready(r0);
+      if (nch > 1) tmem_regs_ready(r1);
+      if (nch > 2) tmem_regs_ready(r2);
+      if (nch > 3) tmem_regs_ready(r3);
       const bool full = nk == KT;
       float mx;
       if (full) {
