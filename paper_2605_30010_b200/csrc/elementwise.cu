@@ -53,31 +53,44 @@ void launch_im2col(const float* frames, void* patches, int T, int image, int pat
 // LayerNorm: one warp per row, row held in registers, mean then centred variance (two passes over
 // registers), fp32 statistics.
 // ---------------------------------------------------------------------------------------------
-template <typename T>
-__global__ void layernorm_kernel(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b,
-                                 float eps, T* __restrict__ y, int rows_cap, int D, const int* __restrict__ n_frames_dev,
-                                 int rows_per_frame) {
+template <typename T, int NV>
+__global__ void __launch_bounds__(256)
+layernorm_kernel(const float* __restrict__ x, const float* __restrict__ g, const float* __restrict__ b, float eps,
+                 T* __restrict__ y, int rows_cap, int D, const int* __restrict__ n_frames_dev, int rows_per_frame) {
   const int rows = n_frames_dev ? min(rows_cap, *n_frames_dev * rows_per_frame) : rows_cap;
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
   for (int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5); row < rows; row += gridDim.x * warps_per_block) {
-    float4 v[ROW_MAX_VEC];
-    load_row(x + (size_t)row * D, D, lane, v);
-    layernorm_row_inplace(v, D, lane, g, b, eps);
-    store_row<T>(y + (size_t)row * D, D, lane, v);
+    float4 v[NV];
+    load_row<NV>(x + (size_t)row * D, D, lane, v);
+    layernorm_row_inplace<NV>(v, D, lane, g, b, eps);
+    store_row<NV>(y + (size_t)row * D, D, lane, v);
   }
+}
+
+template <typename T>
+void launch_layernorm_t(const float* x, const float* g, const float* b, float eps, T* y, int rows_cap, int D,
+                        const int* n_frames_dev, int rows_per_frame, cudaStream_t s) {
+  const int threads = 256, wpb = threads / 32;
+  const int blocks = min(cdiv(rows_cap, wpb), 148 * 16);
+  const int need = cdiv(D / 4, 32);      // float4 chunks per lane: the row lives in exactly that many registers
+#define ET_LN(NV) layernorm_kernel<T, NV><<<blocks, threads, 0, s>>>(x, g, b, eps, y, rows_cap, D, n_frames_dev, rows_per_frame)
+  if (need <= 1) ET_LN(1);
+  else if (need <= 2) ET_LN(2);
+  else if (need <= 4) ET_LN(4);
+  else if (need <= 6) ET_LN(6);
+  else if (need <= 9) ET_LN(9);
+  else if (need <= 12) ET_LN(12);
+  else ET_LN(16);
+#undef ET_LN
 }
 
 void launch_layernorm(const float* x, const float* g, const float* b, float eps, void* y, int rows_cap, int D,
                       bool out_bf16, const int* n_frames_dev, int rows_per_frame, cudaStream_t s) {
   if (rows_cap <= 0) return;
-  const int threads = 256, wpb = threads / 32;
-  const int blocks = min(cdiv(rows_cap, wpb), 148 * 16);
   ET_COUNT_LAUNCH();
-  if (out_bf16)
-    layernorm_kernel<bf16><<<blocks, threads, 0, s>>>(x, g, b, eps, (bf16*)y, rows_cap, D, n_frames_dev, rows_per_frame);
-  else
-    layernorm_kernel<float><<<blocks, threads, 0, s>>>(x, g, b, eps, (float*)y, rows_cap, D, n_frames_dev, rows_per_frame);
+  if (out_bf16) launch_layernorm_t<bf16>(x, g, b, eps, (bf16*)y, rows_cap, D, n_frames_dev, rows_per_frame, s);
+  else launch_layernorm_t<float>(x, g, b, eps, (float*)y, rows_cap, D, n_frames_dev, rows_per_frame, s);
 }
 
 }  // namespace et

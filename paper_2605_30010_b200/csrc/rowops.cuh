@@ -23,38 +23,34 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
-__device__ __forceinline__ void load_row(const float* __restrict__ p, int D, int lane, float4 (&v)[ROW_MAX_VEC]) {
+template <int NV>
+__device__ __forceinline__ void load_row(const float* __restrict__ p, int D, int lane, float4 (&v)[NV]) {
   const int nvec = D >> 2;
   const float4* p4 = reinterpret_cast<const float4*>(p);
 #pragma unroll
-  for (int j = 0; j < ROW_MAX_VEC; ++j) {
+  for (int j = 0; j < NV; ++j) {
     const int i = lane + 32 * j;
     v[j] = (i < nvec) ? __ldg(p4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
 }
 
-template <typename T>
-__device__ __forceinline__ void store_row(T* __restrict__ p, int D, int lane, const float4 (&v)[ROW_MAX_VEC]);
-
-template <>
-__device__ __forceinline__ void store_row<float>(float* __restrict__ p, int D, int lane,
-                                                 const float4 (&v)[ROW_MAX_VEC]) {
+template <int NV>
+__device__ __forceinline__ void store_row(float* __restrict__ p, int D, int lane, const float4 (&v)[NV]) {
   const int nvec = D >> 2;
   float4* p4 = reinterpret_cast<float4*>(p);
 #pragma unroll
-  for (int j = 0; j < ROW_MAX_VEC; ++j) {
+  for (int j = 0; j < NV; ++j) {
     const int i = lane + 32 * j;
     if (i < nvec) p4[i] = v[j];
   }
 }
 
-template <>
-__device__ __forceinline__ void store_row<bf16>(bf16* __restrict__ p, int D, int lane,
-                                                const float4 (&v)[ROW_MAX_VEC]) {
+template <int NV>
+__device__ __forceinline__ void store_row(bf16* __restrict__ p, int D, int lane, const float4 (&v)[NV]) {
   const int nvec = D >> 2;
   uint2* p2 = reinterpret_cast<uint2*>(p);
 #pragma unroll
-  for (int j = 0; j < ROW_MAX_VEC; ++j) {
+  for (int j = 0; j < NV; ++j) {
     const int i = lane + 32 * j;
     if (i < nvec) {
       __nv_bfloat162 lo = __floats2bfloat162_rn(v[j].x, v[j].y);
@@ -68,17 +64,18 @@ __device__ __forceinline__ void store_row<bf16>(bf16* __restrict__ p, int D, int
 }
 
 // y = (x - mean) / sqrt(var + eps) * g + b, statistics in fp32 over the registers of the warp.
-__device__ __forceinline__ void layernorm_row_inplace(float4 (&v)[ROW_MAX_VEC], int D, int lane,
+template <int NV>
+__device__ __forceinline__ void layernorm_row_inplace(float4 (&v)[NV], int D, int lane,
                                                       const float* __restrict__ g, const float* __restrict__ b,
                                                       float eps) {
   const int nvec = D >> 2;
   float s = 0.f;
 #pragma unroll
-  for (int j = 0; j < ROW_MAX_VEC; ++j) s += (v[j].x + v[j].y) + (v[j].z + v[j].w);   // padding chunks are zero
+  for (int j = 0; j < NV; ++j) s += (v[j].x + v[j].y) + (v[j].z + v[j].w);   // padding chunks are zero
   const float mean = warp_sum(s) / (float)D;
   float q = 0.f;
 #pragma unroll
-  for (int j = 0; j < ROW_MAX_VEC; ++j) {
+  for (int j = 0; j < NV; ++j) {
     if (lane + 32 * j < nvec) {
       const float a = v[j].x - mean, c = v[j].y - mean, d = v[j].z - mean, e = v[j].w - mean;
       q += (a * a + c * c) + (d * d + e * e);
@@ -88,7 +85,7 @@ __device__ __forceinline__ void layernorm_row_inplace(float4 (&v)[ROW_MAX_VEC], 
   const float4* g4 = reinterpret_cast<const float4*>(g);
   const float4* b4 = reinterpret_cast<const float4*>(b);
 #pragma unroll
-  for (int j = 0; j < ROW_MAX_VEC; ++j) {
+  for (int j = 0; j < NV; ++j) {
     const int i = lane + 32 * j;
     if (i < nvec) {
       const float4 gg = __ldg(g4 + i), bb = __ldg(b4 + i);

@@ -208,9 +208,9 @@ gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restric
   for (int r = blockIdx.x * nwarps + wid; r < kept; r += gridDim.x * nwarps) {
     const int j = sh_pos[r];
     float4 v[ROW_MAX_VEC];
-    load_row(x + ((size_t)f * L + j) * D, D, lane, v);
-    if (ln_g) layernorm_row_inplace(v, D, lane, ln_g, ln_b, eps);
-    store_row<float>(tokens + (size_t)(out0 + r) * D, D, lane, v);
+    load_row<ROW_MAX_VEC>(x + ((size_t)f * L + j) * D, D, lane, v);
+    if (ln_g) layernorm_row_inplace<ROW_MAX_VEC>(v, D, lane, ln_g, ln_b, eps);
+    store_row<ROW_MAX_VEC>(tokens + (size_t)(out0 + r) * D, D, lane, v);
     if (lane == 0) token_pos[out0 + r] = j;
   }
 }
