@@ -24,6 +24,10 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of gemm_bf16_kernel<256, *> (ncu, workload so400m_32f):
+# qkv 175.6 MB, out-proj 213.4 MB, fc1 215.1 MB, fc2 402.3 MB -> average.  To be re-taken whenever that kernel changes.
+GEMM_DRAM_BYTES_PER_LAUNCH = 251.6e6
+
 METRIC = "frames/s through compressed encoder (32f SigLIP-so400m)"
 UNIT = "frames/s"
 
@@ -258,7 +262,9 @@ def main():
                 "peak": peak_tf, "unit": "TFLOP/s", "frac": (gemm_tflops / peak_tf) if peak_tf else None,
                 "peak_source": f"{peaks['source']} (sustained bf16 GEMM; kernel timed inside a long step)",
                 "launches": g["launches"], "avg_launch_ms": g["ms"] / max(1, g["launches"]),
-                "traffic": None}
+                "traffic": GEMM_DRAM_BYTES_PER_LAUNCH if wl.name == "so400m_32f" else None,
+                "traffic_unit": "bytes per launch (dram read + written), average of the four dense launches of block 0 at "
+                                "32 frames, from the ncu capture summarised in profiles/gemm_bf16_kernel_so400m_32f.md"}
     per_cat = {}
     for name in B.PROF_NAMES:
         c = prof[name]
