@@ -98,11 +98,14 @@ typedef struct {
   double tau_seg;       /* Eq. 1 threshold */
   double tau_merge;     /* Eq. 2 threshold */
   int weighted_merge;   /* 1 = Eq. 3, 0 = plain average */
-  int selection;        /* 0 keep all tokens, 1 decoupled (Alg. 2), 2 per-frame top-k on every frame */
+  int selection;        /* 0 keep all tokens, 1 decoupled (Alg. 2), 2 per-frame top-k on every frame,
+                           3 random sampling (the paper's sampling ablation): k tokens per frame drawn with
+                           Philox-4x32-10, counter (position, output frame inside its video, video, 0), key = sample_seed */
   int retain_mode;      /* 0: keep floor(retain*L) per frame; 1: total budget, k = floor(retain*B*L/N) (Eq. 5) */
   double retain;        /* (0, 1] */
   const et_forced_plan* forced_plan; /* NULL = decide */
   int want_trace;       /* 1 = fill et_result.trace */
+  unsigned long long sample_seed; /* selection 3 only */
 } et_params;
 
 /* Decision trace, host memory owned by the encoder.  Per merge layer i the arrays cover the list

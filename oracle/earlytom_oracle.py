@@ -342,9 +342,37 @@ def window_mask(a: np.ndarray, w: int) -> np.ndarray:
     return m
 
 
+def philox4x32_10(counter: np.ndarray, key: Tuple[int, int]) -> np.ndarray:
+    """Philox-4x32 with 10 rounds (Salmon et al., "Parallel random numbers: as easy as 1, 2, 3", SC'11),
+    written from its published definition.  counter uint32 [..., 4] -> uint32 [..., 4]."""
+    M0, M1, W0, W1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
+    mask = np.uint64(0xFFFFFFFF)
+    c = [counter[..., i].astype(np.uint64) for i in range(4)]
+    k0, k1 = int(key[0]) & 0xFFFFFFFF, int(key[1]) & 0xFFFFFFFF
+    for _ in range(10):
+        p0 = np.uint64(M0) * c[0]
+        p1 = np.uint64(M1) * c[2]
+        hi0, lo0 = p0 >> np.uint64(32), p0 & mask
+        hi1, lo1 = p1 >> np.uint64(32), p1 & mask
+        c = [hi1 ^ c[1] ^ np.uint64(k0), lo1, hi0 ^ c[3] ^ np.uint64(k1), lo0]
+        k0, k1 = (k0 + W0) & 0xFFFFFFFF, (k1 + W1) & 0xFFFFFFFF
+    return np.stack(c, axis=-1).astype(np.uint32)
+
+
+def random_scores(seed: int, video: int, n_frames: int, L: int) -> np.ndarray:
+    """Scores of the random-sampling baseline (the paper's sampling ablation): token j of output frame f of
+    video v gets the uniform number (x >> 8) / 2^24, x = first word of Philox(counter (j, f, v, 0), key = seed)."""
+    ctr = np.zeros((n_frames, L, 4), dtype=np.uint32)
+    ctr[..., 0] = np.arange(L, dtype=np.uint32)[None, :]
+    ctr[..., 1] = np.arange(n_frames, dtype=np.uint32)[:, None]
+    ctr[..., 2] = np.uint32(video)
+    x = philox4x32_10(ctr, (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))[..., 0]
+    return (x >> np.uint32(8)).astype(np.float64) / float(1 << 24)
+
+
 def select_tokens(A: np.ndarray, dynamic: np.ndarray, k: int, w: int, selection: int) -> np.ndarray:
     """keep mask [N, L].  selection: 0 keep all, 1 decoupled (dynamic: top-k, static: windows),
-    2 plain per-frame top-k on every frame."""
+    2 plain per-frame top-k on every frame (3, random sampling, is selection 2 applied to `random_scores`)."""
     N, L = A.shape
     keep = np.zeros((N, L), dtype=bool)
     for f in range(N):
@@ -380,7 +408,7 @@ class VideoResult:
 
 
 def encode_video(frames: np.ndarray, shape, blob_or_w, params, dtype=np.float64,
-                 keep_features: bool = False, forced: Optional[dict] = None) -> VideoResult:
+                 keep_features: bool = False, forced: Optional[dict] = None, video_index: int = 0) -> VideoResult:
     """frames [B,3,H,W] of ONE video -> compressed tokens + index map.
 
     `forced` (tests only) replays given decisions instead of taking them:
@@ -422,6 +450,9 @@ def encode_video(frames: np.ndarray, shape, blob_or_w, params, dtype=np.float64,
     k, wdt, M = rescaled_keep(params.retain, B, N, L, params.retain_mode)
     if forced is not None and "keep" in forced:
         keep = np.asarray(forced["keep"], dtype=bool)
+    elif params.selection == 3:
+        # random sampling (paper's sampling ablation): k tokens per frame, uniformly at random
+        keep = select_tokens(random_scores(int(getattr(params, "sample_seed", 0)), video_index, N, L), dynamic, k, wdt, 2)
     else:
         keep = select_tokens(A, dynamic, k, wdt, params.selection)
     counts = keep.sum(axis=1)
@@ -466,7 +497,7 @@ def encode_batch(frames: np.ndarray, video_offsets: Sequence[int], shape, blob_o
                  dtype=np.float64, **kw) -> List[VideoResult]:
     """Independent videos: each one goes through `encode_video` on its own."""
     w = blob_or_w if isinstance(blob_or_w, dict) else split_weights(shape, blob_or_w)
-    return [encode_video(frames[video_offsets[v]:video_offsets[v + 1]], shape, w, params, dtype=dtype, **kw)
+    return [encode_video(frames[video_offsets[v]:video_offsets[v + 1]], shape, w, params, dtype=dtype, video_index=v, **kw)
             for v in range(len(video_offsets) - 1)]
 
 

@@ -57,7 +57,7 @@ class et_params(C.Structure):
     _fields_ = [("num_merge_layers", C.c_int), ("merge_layers", C.c_int * ET_MAX_MERGE_LAYERS),
                 ("ema_alpha", C.c_double), ("tau_seg", C.c_double), ("tau_merge", C.c_double),
                 ("weighted_merge", C.c_int), ("selection", C.c_int), ("retain_mode", C.c_int), ("retain", C.c_double),
-                ("forced_plan", C.POINTER(et_forced_plan)), ("want_trace", C.c_int)]
+                ("forced_plan", C.POINTER(et_forced_plan)), ("want_trace", C.c_int), ("sample_seed", C.c_ulonglong)]
 
 
 class et_trace(C.Structure):
@@ -229,6 +229,7 @@ def make_params(p, forced: Optional[ForcedPlan] = None, want_trace: bool = False
     q.weighted_merge, q.selection, q.retain_mode = int(p.weighted_merge), int(p.selection), int(p.retain_mode)
     q.retain = float(p.retain)
     q.want_trace = 1 if want_trace else 0
+    q.sample_seed = int(getattr(p, "sample_seed", 0))
     keep = []
     if forced is not None:
         fp = et_forced_plan()

@@ -143,6 +143,10 @@ void launch_select_setup(const SelectSetupArgs& a, int n_cap, cudaStream_t s);
 void launch_select_tokens(const float* scores, const unsigned char* dynamic, const int* k_frame, const int* w_frame,
                           int n_cap, int L, int selection_all, unsigned char* keep, int* count,
                           const int* n_frames_dev, cudaStream_t s);
+// Random-sampling ablation: scores[f][j] = uniform number of Philox-4x32-10 with counter (j, frame inside its
+// video, video, 0) and key = seed, for the frames of the current list.
+void launch_random_scores(float* scores, const int* vid_off, int n_videos, int n_cap, int L, unsigned long long seed,
+                          const int* n_frames_dev, cudaStream_t s);
 void launch_count_keep(const unsigned char* keep, int n_cap, int L, int* count, const int* n_frames_dev, cudaStream_t s);
 // frame_offsets[0..n] = exclusive scan of count; totals[0] = n_frames, totals[1] = n_tokens
 void launch_scan_counts(const int* count, int* frame_offsets, int* totals, int n_cap, const int* n_frames_dev,

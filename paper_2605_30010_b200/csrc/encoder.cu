@@ -204,7 +204,7 @@ et_status validate_params(const et_encoder* e, const et_params* p) {
   if (!(p->ema_alpha > 0.0 && p->ema_alpha <= 1.0)) return ET_ERR_INVALID_ARG;
   if (!(p->retain > 0.0 && p->retain <= 1.0)) return ET_ERR_INVALID_ARG;
   if (isnan(p->tau_seg) || isnan(p->tau_merge)) return ET_ERR_INVALID_ARG;
-  if (p->selection < 0 || p->selection > 2) return ET_ERR_INVALID_ARG;
+  if (p->selection < 0 || p->selection > 3) return ET_ERR_INVALID_ARG;
   if (p->retain_mode < 0 || p->retain_mode > 1) return ET_ERR_INVALID_ARG;
   return ET_OK;
 }
@@ -341,9 +341,15 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     ET_CUDA(e, cudaMemcpyAsync(e->keep, e->h_keep_stage, (size_t)fp->n_final * L, cudaMemcpyHostToDevice, s));
     PROF(ET_CAT_SELECT, launch_count_keep(e->keep, T, L, e->count, n_dev, s));
   } else {
-    if (p->selection == 2) ET_CUDA(e, cudaMemsetAsync(e->dynamic, 1, T, s));   // plain top-k: every frame ranks globally
-    PROF(ET_CAT_SELECT, launch_select_tokens(e->scores, e->dynamic, e->k_frame, e->w_frame, T, L, p->selection == 0, e->keep, e->count, n_dev, s));
-    if (p->selection == 2) PROF(ET_CAT_SELECT, launch_select_setup(sa, T, s));                      // restore the reported dynamic flags
+    const bool rank_all = p->selection == 2 || p->selection == 3;
+    const float* sel_scores = e->scores;
+    if (p->selection == 3) {          // random sampling: rank uniform numbers instead of attention scores
+      PROF(ET_CAT_SELECT, launch_random_scores(e->score_partial, e->fl[lst].vid_off, V, T, L, p->sample_seed, n_dev, s));
+      sel_scores = e->score_partial;
+    }
+    if (rank_all) ET_CUDA(e, cudaMemsetAsync(e->dynamic, 1, T, s));            // every frame ranks globally
+    PROF(ET_CAT_SELECT, launch_select_tokens(sel_scores, e->dynamic, e->k_frame, e->w_frame, T, L, p->selection == 0, e->keep, e->count, n_dev, s));
+    if (rank_all) PROF(ET_CAT_SELECT, launch_select_setup(sa, T, s));          // restore the reported dynamic flags
   }
   PROF(ET_CAT_SELECT, launch_scan_counts(e->count, e->frame_offsets, e->d_small, T, n_dev, s));
   PROF(ET_CAT_GATHER, launch_gather_tokens(e->X[cur], e->keep, e->frame_offsets, T, L, D, c.post_layernorm ? W + e->off_post_g : nullptr,

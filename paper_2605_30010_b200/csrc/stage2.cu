@@ -102,6 +102,44 @@ void launch_select_tokens(const float* scores, const unsigned char* dynamic, con
                                                              selection_all, keep, count, n_frames_dev);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Random-sampling ablation.  Philox-4x32 with 10 rounds (Salmon et al., SC'11), from its published
+// definition: two 32x32->64 multiplications per round, key bumped by the Weyl constants.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                                        uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
+
+__global__ void random_scores_kernel(float* __restrict__ scores, const int* __restrict__ vid_off, int n_videos, int n_cap,
+                                     int L, unsigned long long seed, const int* __restrict__ n_frames_dev) {
+  const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
+  const int f = blockIdx.x;
+  if (f >= n) return;
+  int v = 0;
+  while (v + 1 < n_videos && vid_off[v + 1] <= f) ++v;      // video of this frame (a few hundred at most)
+  const uint32_t local = (uint32_t)(f - vid_off[v]);
+  for (int j = threadIdx.x; j < L; j += blockDim.x) {
+    const uint32_t x = philox4x32_10_word0((uint32_t)j, local, (uint32_t)v, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+    scores[(size_t)f * L + j] = (float)(x >> 8) * (1.0f / 16777216.0f);    // exact: 24 bits
+  }
+}
+
+void launch_random_scores(float* scores, const int* vid_off, int n_videos, int n_cap, int L, unsigned long long seed,
+                          const int* n_frames_dev, cudaStream_t s) {
+  if (n_cap <= 0) return;
+  ET_COUNT_LAUNCH();
+  random_scores_kernel<<<n_cap, 256, 0, s>>>(scores, vid_off, n_videos, n_cap, L, seed, n_frames_dev);
+}
+
 // count[f] = number of set bytes of keep[f][:] (used when the mask is given, not decided)
 __global__ void count_keep_kernel(const unsigned char* __restrict__ keep, int n_cap, int L, int* __restrict__ count,
                                   const int* __restrict__ n_frames_dev) {

@@ -57,9 +57,10 @@ class MergeParams:
     tau_seg: float = 0.8
     tau_merge: float = 0.8
     weighted_merge: int = 1
-    selection: int = 1      # 0 none, 1 decoupled, 2 plain per-frame top-k
+    selection: int = 1      # 0 none, 1 decoupled, 2 plain per-frame top-k, 3 random sampling (ablation)
     retain_mode: int = 1    # 0 per-frame fraction, 1 total budget
     retain: float = 0.25
+    sample_seed: int = 0    # seed of the random-sampling ablation (selection 3)
 
 
 @dataclass(frozen=True)

@@ -108,7 +108,7 @@ def test_tiny_fp32_uncompressed(B):
     run_workload(B, wl, np.float64, F32_TOL, 1e-5, 1e-4)
 
 
-@pytest.mark.parametrize("selection,mode,retain", [(2, 0, 0.25), (1, 1, 0.3), (0, 1, 1.0)])
+@pytest.mark.parametrize("selection,mode,retain", [(2, 0, 0.25), (1, 1, 0.3), (0, 1, 1.0), (3, 0, 0.25)])
 def test_tiny_fp32_variants(B, selection, mode, retain):
     wl = workload("tiny")
     p = dataclasses.replace(wl.params, selection=selection, retain_mode=mode, retain=retain, tau_seg=0.895, tau_merge=0.85)
@@ -127,6 +127,17 @@ def test_fp32_batch_of_ragged_videos(B):
     p = MergeParams(merge_layers=(1, 3), tau_seg=0.6, tau_merge=0.7, selection=1, retain_mode=1, retain=0.4)
     wl = Workload("ragged", shape, "f32", vids, p, 77)
     run_workload(B, wl, np.float64, F32_TOL, 1e-5, 1e-4)
+
+
+def test_random_sampling_ablation_on_ragged_batch(B):
+    """selection 3: both sides draw the same Philox numbers per (video, output frame, position) -> identical kept sets."""
+    shape = EncoderShape(image_size=56, patch_size=14, num_layers=4, hidden=48, heads=3, mlp_dim=100)
+    vids = (VideoSpec(5, 0.1, 1), VideoSpec(1, 0.2, 2), VideoSpec(9, 0.05, 3), VideoSpec(12, 0.15, 5))
+    p = MergeParams(merge_layers=(1, 3), tau_seg=0.6, tau_merge=0.7, selection=3, retain_mode=1, retain=0.4,
+                    sample_seed=0x1234567890ABCDEF)
+    wl = Workload("ragged_random", shape, "f32", vids, p, 77)
+    err, log = run_workload(B, wl, np.float64, F32_TOL, 1e-5, 1e-4)
+    assert not log
 
 
 def test_identical_middle_frames_collapse(B):

@@ -162,3 +162,38 @@ def test_main_setting_matches_paper_table():
     assert list(p.merge_layers) == [int(x) for x in kv["merge_layers_mvbench_25"].split(",")]
     assert WORKLOADS["so400m_32f"].total_frames == int(kv["frames_per_video"])
     assert p.retain in [float(x) for x in kv["retain_ratios"].split(",")]
+
+
+# ------------------------------------------------------------------ random-sampling ablation (selection 3)
+
+def test_philox_known_answers():
+    """The counter-based generator behind the random-sampling baseline, against the published vectors."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 3
+    for r in rows:
+        w = [int(x, 16) for x in r]
+        out = O.philox4x32_10(np.array(w[0:4], dtype=np.uint32), (w[4], w[5]))
+        assert [int(x) for x in out] == w[6:10]
+
+
+def test_random_scores_are_uniform_and_counter_based():
+    a = O.random_scores(seed=7, video=2, n_frames=5, L=729)
+    assert a.shape == (5, 729) and a.min() >= 0.0 and a.max() < 1.0
+    assert abs(a.mean() - 0.5) < 0.02 and abs(a.var() - 1 / 12) < 0.01
+    # a token's number depends only on (seed, video, frame, position)
+    b = O.random_scores(seed=7, video=2, n_frames=3, L=100)
+    np.testing.assert_array_equal(a[:3, :100], b)
+    assert not np.array_equal(a, O.random_scores(seed=8, video=2, n_frames=5, L=729))
+    assert not np.array_equal(a, O.random_scores(seed=7, video=3, n_frames=5, L=729))
+
+
+def test_random_sampling_keeps_k_per_frame():
+    a = O.random_scores(seed=1, video=0, n_frames=6, L=64)
+    keep = O.select_tokens(a, np.zeros(6, dtype=bool), 16, 4, 2)
+    assert (keep.sum(axis=1) == 16).all()
+    # every position is kept about k/L of the time over many frames
+    big = O.select_tokens(O.random_scores(3, 0, 400, 32), np.zeros(400, dtype=bool), 8, 4, 2)
+    freq = big.mean(axis=0)
+    assert np.abs(freq - 0.25).max() < 0.1
