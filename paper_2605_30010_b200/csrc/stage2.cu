@@ -217,6 +217,7 @@ void launch_scan_counts(const int* count, int* frame_offsets, int* totals, int n
 // ---------------------------------------------------------------------------------------------
 constexpr int GATHER_MAX_L = 4096;
 
+template <int NV>
 __global__ void __launch_bounds__(256)
 gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restrict__ keep,
                      const int* __restrict__ frame_offsets, int n_cap, int L, int D, const float* __restrict__ ln_g,
@@ -245,10 +246,10 @@ gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restric
   const int out0 = frame_offsets[f];
   for (int r = blockIdx.x * nwarps + wid; r < kept; r += gridDim.x * nwarps) {
     const int j = sh_pos[r];
-    float4 v[ROW_MAX_VEC];
-    load_row<ROW_MAX_VEC>(x + ((size_t)f * L + j) * D, D, lane, v);
-    if (ln_g) layernorm_row_inplace<ROW_MAX_VEC>(v, D, lane, ln_g, ln_b, eps);
-    store_row<ROW_MAX_VEC>(tokens + (size_t)(out0 + r) * D, D, lane, v);
+    float4 v[NV];
+    load_row<NV>(x + ((size_t)f * L + j) * D, D, lane, v);
+    if (ln_g) layernorm_row_inplace<NV>(v, D, lane, ln_g, ln_b, eps);
+    store_row<NV>(tokens + (size_t)(out0 + r) * D, D, lane, v);
     if (lane == 0) token_pos[out0 + r] = j;
   }
 }
@@ -259,8 +260,17 @@ void launch_gather_tokens(const float* x, const unsigned char* keep, const int* 
   if (n_cap <= 0) return;
   const int slices = max(1, min(16, cdiv(L, 64)));
   ET_COUNT_LAUNCH();
-  gather_tokens_kernel<<<dim3(slices, n_cap), 256, sizeof(unsigned short) * L, s>>>(
-      x, keep, frame_offsets, n_cap, L, D, ln_g, ln_b, eps, tokens, token_pos, n_frames_dev);
+  const int need = cdiv(D / 4, 32);      // float4 chunks per lane
+#define ET_GATHER(NV)                                                                                      \
+  gather_tokens_kernel<NV><<<dim3(slices, n_cap), 256, sizeof(unsigned short) * L, s>>>(                   \
+      x, keep, frame_offsets, n_cap, L, D, ln_g, ln_b, eps, tokens, token_pos, n_frames_dev)
+  if (need <= 2) ET_GATHER(2);
+  else if (need <= 4) ET_GATHER(4);
+  else if (need <= 6) ET_GATHER(6);
+  else if (need <= 9) ET_GATHER(9);
+  else if (need <= 12) ET_GATHER(12);
+  else ET_GATHER(16);
+#undef ET_GATHER
 }
 
 }  // namespace et
