@@ -89,24 +89,8 @@ __device__ __forceinline__ float row_max(const uint32_t (&r)[32], int c0, int nk
   return fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
 }
 
-// Packed fp32 pairs (one instruction for two elements on sm_100).  The exponential phase of the softmax is bound by
-// instruction issue: halving the FMA and ADD count is worth 4 % of the kernel; a three-input maximum and a cubic
-// exp2 on the FMA pipe were measured slower.
-__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {
-  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
-      "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
-      "mov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
-}
-__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
-  asm("{\n\t.reg .b64 ra, rd;\n\t"
-      "mov.b64 ra, {%2, %3};\n\tmov.b64 rd, {%0, %1};\n\t"
-      "add.rn.f32x2 rd, rd, ra;\n\t"
-      "mov.b64 {%0, %1}, rd;\n\t}"
-      : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
-}
-
+// The exponential phase of the softmax is bound by instruction issue: packed fp32 pairs (fma2 / add2) halve the FMA
+// and ADD count, worth 4 % of the kernel; a three-input maximum and a cubic exp2 on the FMA pipe were measured slower.
 template <bool MASK>
 __device__ __forceinline__ void probs(const uint32_t (&r)[32], int c0, int nk, float scale2, float m, float (&ls)[4],
                                       uint32_t p_addr) {
@@ -115,14 +99,14 @@ __device__ __forceinline__ void probs(const uint32_t (&r)[32], int c0, int nk, f
 #pragma unroll
   for (int i = 0; i < 32; i += 2) {
     float x0, x1;
-    fma2(x0, x1, __uint_as_float(r[i]), __uint_as_float(r[i + 1]), scale2, neg_m);
+    fma2(x0, x1, __uint_as_float(r[i]), __uint_as_float(r[i + 1]), scale2, scale2, neg_m, neg_m);
     float p0 = ex2(x0), p1 = ex2(x1);
     if (MASK) {
       if (c0 + i >= nk) p0 = 0.f;
       if (c0 + i + 1 >= nk) p1 = 0.f;
     }
     const int a = ((i >> 1) & 1) * 2;                // two pairs of partial sums, alternating
-    add2(ls[a], ls[a + 1], p0, p1);
+    add2(ls[a], ls[a + 1], ls[a], ls[a + 1], p0, p1);
     pk[i >> 1] = pack_bf16(p0, p1);
   }
   tmem_st16(p_addr, pk);

@@ -146,6 +146,16 @@ __device__ __forceinline__ float gelu_tanh_fast(float x) {
   const float hx = 0.5f * x;
   return fmaf(hx, tanh_fast(inner), hx);
 }
+// The same on two elements with packed instructions (identical operations per element, hence identical bits).
+__device__ __forceinline__ void gelu_tanh_fast2(float& x0, float& x1) {
+  const float c = 0.7978845608028654f, k = 0.044715f * c;
+  float u0, u1, t0, t1, i0, i1, h0, h1;
+  mul2(u0, u1, x0, x1, x0, x1);
+  fma2(t0, t1, u0, u1, k, k, c, c);
+  mul2(i0, i1, x0, x1, t0, t1);
+  mul2(h0, h1, x0, x1, 0.5f, 0.5f);
+  fma2(x0, x1, h0, h1, tanh_fast(i0), tanh_fast(i1), h0, h1);
+}
 // Both store paths of the epilogue go through this function, so a row gets the same bits whichever path writes it.
 __device__ __forceinline__ float gelu_epi(float x, int tanh_approx) {
   if (tanh_approx) return gelu_tanh_fast(x);
@@ -303,13 +313,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
             float v[32];
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
-              v[q * 4 + 0] = __uint_as_float(r[q * 4 + 0]) + b[q].x; v[q * 4 + 1] = __uint_as_float(r[q * 4 + 1]) + b[q].y;
-              v[q * 4 + 2] = __uint_as_float(r[q * 4 + 2]) + b[q].z; v[q * 4 + 3] = __uint_as_float(r[q * 4 + 3]) + b[q].w;
+              add2(v[q * 4 + 0], v[q * 4 + 1], __uint_as_float(r[q * 4 + 0]), __uint_as_float(r[q * 4 + 1]), b[q].x, b[q].y);
+              add2(v[q * 4 + 2], v[q * 4 + 3], __uint_as_float(r[q * 4 + 2]), __uint_as_float(r[q * 4 + 3]), b[q].z, b[q].w);
             }
             if (EPI == EPI_GELU) {
               if (g.gelu_tanh) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = gelu_tanh_fast(v[i]);
+                for (int i = 0; i < 32; i += 2) gelu_tanh_fast2(v[i], v[i + 1]);
               } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = gelu_epi(v[i], 0);
