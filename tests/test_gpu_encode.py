@@ -141,7 +141,7 @@ def test_random_sampling_ablation_on_ragged_batch(B):
 
 
 def test_identical_middle_frames_collapse(B):
-    """[H, X, X, Y, T]: the two identical frames merge into one frame equal to X (spec self-check)."""
+    """[H, X, X, Y, T]: the two identical frames merge into one frame equal to X."""
     wl = workload("tiny")
     v = make_video(5, 112, 14, 0.6, seed=3)
     v[2] = v[1]
