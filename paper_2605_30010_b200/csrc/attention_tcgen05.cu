@@ -428,6 +428,12 @@ cudaError_t run(const AttnMaps& maps, const AttnArgs& a, cudaStream_t s) {
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES);
     if (e != cudaSuccess) return e;
+    // setmaxnreg.inc waits for registers that only exist if the kernel was compiled with at least LAUNCH_REGS per
+    // thread: refuse to launch (instead of blocking for ever) should a compiler ever assign fewer.
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, attention_tc_kernel<DH>);
+    if (e != cudaSuccess) return e;
+    if (fa.numRegs < LAUNCH_REGS) return cudaErrorLaunchOutOfResources;
     configured = true;
   }
   ET_COUNT_LAUNCH();
