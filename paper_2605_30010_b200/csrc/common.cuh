@@ -72,6 +72,10 @@ struct TmaDesc { alignas(64) unsigned char bytes[128]; };
 // Build a 2-D bf16 tensor map: rows x cols (cols contiguous), box box_rows x 64 cols, 128-byte swizzle.
 bool make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
                       const char** err);
+// Weight operand w [N][K]: one map whose box holds a CTA's half of a full-width tile, one with a 64-row box for
+// the narrow last column tile (N mod 256 <= 128), so that a narrow tile does not fetch weight rows it never uses.
+struct WeightDesc { TmaDesc full, half; };
+bool make_tma_weight(WeightDesc* out, const void* base, uint64_t n_rows, uint64_t k_cols, const char** err);
 // Tensor map of a dense layer's output c [rows][cols] (fp32 or bf16): 32 x 32 boxes for the epilogue's
 // TMA stores / reduce-adds.
 bool make_tma_out(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, bool fp32, const char** err);
@@ -79,8 +83,8 @@ int gemm_bf16_pick_bn(int N);
 // Rows of the w box: each CTA of a pair loads half of the tile's BN weight rows.
 int gemm_bf16_w_box_rows(int N);
 // c = epi(a[M][K] * w[N][K]^T + bias).  Descriptors must have been built for (a: M_cap x K, box 128),
-// (w: N x K, box = gemm_bf16_w_box_rows(N)) and (c: make_tma_out; unused by EPI_TABLE).
-cudaError_t launch_gemm_bf16(const TmaDesc& da, const TmaDesc& dw, const TmaDesc& dc, const float* bias, void* c,
+// (w: make_tma_weight) and (c: make_tma_out; unused by EPI_TABLE).
+cudaError_t launch_gemm_bf16(const TmaDesc& da, const WeightDesc& dw, const TmaDesc& dc, const float* bias, void* c,
                              int M_cap, int N, int K, int epilogue, int gelu_tanh, const float* table, int table_rows,
                              const int* n_frames_dev, int rows_per_frame, int* status_dev, cudaStream_t s);
 

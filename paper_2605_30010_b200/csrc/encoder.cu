@@ -38,7 +38,7 @@ struct LayerOffsets { size_t ln1_g, ln1_b, wqkv, bqkv, wo, bo, ln2_g, ln2_b, w1,
 
 struct LayerBf16 {
   bf16 *wqkv_t, *wo_t, *w1_t, *w2_t;
-  TmaDesc d_wqkv, d_wo, d_w1, d_w2;
+  WeightDesc d_wqkv, d_wo, d_w1, d_w2;
 };
 
 }  // namespace
@@ -59,7 +59,7 @@ struct et_encoder {
   size_t off_patch_w = 0, off_patch_b = 0, off_pos = 0, off_post_g = 0, off_post_b = 0;
   std::vector<LayerOffsets> lo;
   bf16* patch_w_t = nullptr;
-  TmaDesc d_patch_w;
+  WeightDesc d_patch_w;
   std::vector<LayerBf16> lb;
 
   // activations
@@ -210,7 +210,7 @@ et_status validate_params(const et_encoder* e, const et_params* p) {
 }
 
 // One dense layer of the encoder on the arithmetic path the encoder was created with.
-et_status dense(et_encoder* e, const void* a, const TmaDesc& da, const float* w_f32, const TmaDesc& dw,
+et_status dense(et_encoder* e, const void* a, const TmaDesc& da, const float* w_f32, const WeightDesc& dw,
                 const TmaDesc& dc, const float* bias, void* c, int M_cap, int N, int K, int epi, const float* table, int table_rows,
                 const int* n_dev, cudaStream_t s) {
   if (e->bf) {
@@ -296,7 +296,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     const int* n_dev = e->fl[lst].n;
     const LayerOffsets& o = e->lo[layer];
     const LayerBf16* b = e->bf ? &e->lb[layer] : nullptr;
-    static const TmaDesc none{};
+    static const WeightDesc none{};
     PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln1_g, W + o.ln1_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
     PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.wqkv, b ? b->d_wqkv : none, e->c_QKV, W + o.bqkv, e->QKV, rows_cap, 3 * D, D, EPI_STORE,
                  nullptr, 1, n_dev, s)));
@@ -532,7 +532,7 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
       return cudaGetLastError() == cudaSuccess ? ET_OK : ET_ERR_CUDA;
     };
     if ((st = convert(e->off_patch_w, P, (int)D, e->Kp, &e->patch_w_t)) != ET_OK) return bail(st);
-    if (!make_tma_2d_bf16(&e->d_patch_w, e->patch_w_t, D, e->Kp, gemm_bf16_w_box_rows((int)D), &err)) return bail(fail(e, ET_ERR_CUDA, err));
+    if (!make_tma_weight(&e->d_patch_w, e->patch_w_t, D, e->Kp, &err)) return bail(fail(e, ET_ERR_CUDA, err));
     e->lb.resize(config->num_layers);
     for (int i = 0; i < config->num_layers; ++i) {
       LayerBf16& b = e->lb[i];
@@ -541,10 +541,10 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
       if ((st = convert(o.wo, (int)D, (int)D, (int)D, &b.wo_t)) != ET_OK) return bail(st);
       if ((st = convert(o.w1, (int)D, (int)M, (int)D, &b.w1_t)) != ET_OK) return bail(st);
       if ((st = convert(o.w2, (int)M, (int)D, (int)M, &b.w2_t)) != ET_OK) return bail(st);
-      bool ok = make_tma_2d_bf16(&b.d_wqkv, b.wqkv_t, 3 * D, D, gemm_bf16_w_box_rows((int)(3 * D)), &err) &&
-                make_tma_2d_bf16(&b.d_wo, b.wo_t, D, D, gemm_bf16_w_box_rows((int)D), &err) &&
-                make_tma_2d_bf16(&b.d_w1, b.w1_t, M, D, gemm_bf16_w_box_rows((int)M), &err) &&
-                make_tma_2d_bf16(&b.d_w2, b.w2_t, D, M, gemm_bf16_w_box_rows((int)D), &err);
+      bool ok = make_tma_weight(&b.d_wqkv, b.wqkv_t, 3 * D, D, &err) &&
+                make_tma_weight(&b.d_wo, b.wo_t, D, D, &err) &&
+                make_tma_weight(&b.d_w1, b.w1_t, M, D, &err) &&
+                make_tma_weight(&b.d_w2, b.w2_t, D, M, &err);
       if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
     }
     bool ok = make_tma_2d_bf16(&e->d_Pm, e->Pm, rows, e->Kp, 128, &err) && make_tma_2d_bf16(&e->d_Xn, e->Xn, rows, D, 128, &err) &&
@@ -748,9 +748,10 @@ et_status et_linear_bf16(const void* a_dev, const void* w_dev, const float* bias
   if (!a_dev || !w_dev || !bias_dev || !c_dev) return ET_ERR_INVALID_ARG;
   if (M < 1 || N < 8 || N % 8 != 0 || K < 8 || K % 8 != 0) return ET_ERR_SHAPE;
   if (epilogue < 0 || epilogue > 3 || (epilogue == 3 && (!table_dev || table_rows < 1))) return ET_ERR_INVALID_ARG;
-  TmaDesc da, dw, dc;
+  TmaDesc da, dc;
+  WeightDesc dw;
   const char* err = nullptr;
-  if (!make_tma_2d_bf16(&da, a_dev, M, K, 128, &err) || !make_tma_2d_bf16(&dw, w_dev, N, K, gemm_bf16_w_box_rows(N), &err) ||
+  if (!make_tma_2d_bf16(&da, a_dev, M, K, 128, &err) || !make_tma_weight(&dw, w_dev, N, K, &err) ||
       !make_tma_out(&dc, c_dev, M, N, epilogue >= 2, &err))
     return ET_ERR_CUDA;
   ET_CUDA0(launch_gemm_bf16(da, dw, dc, bias_dev, c_dev, M, N, K, epilogue, gelu_tanh, table_dev, table_rows, nullptr, 1,

@@ -169,6 +169,7 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 template <int BN, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b,
+                 const __grid_constant__ CUtensorMap tma_bh,
                  const __grid_constant__ CUtensorMap tma_c, GemmArgs g) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
@@ -218,20 +219,26 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_a) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_b) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_bh) : "memory");
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
         const int m0 = (tile / tiles_n) * (BM * CG) + (int)rank * BM;
-        const int n0 = (tile % tiles_n) * BN + (int)rank * C::B_ROWS;
+        // A last column tile of at most 128 valid columns is multiplied at that width: each CTA then holds 64 weight
+        // rows, fetched through the 64-row box.
+        const int nt0 = (tile % tiles_n) * BN;
+        const bool narrow = BN == 256 && g.N - nt0 <= 128;
+        const int n0 = nt0 + (int)rank * (narrow ? 64 : C::B_ROWS);
+        const uint32_t stage_tx = narrow ? (uint32_t)(C::A_BYTES + 64 * BK * 2) : (uint32_t)C::STAGE_BYTES;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
           const uint32_t full_leader = map_to_cta(full_bar(stage), 0);
           // the leader's barrier counts the bytes of both CTAs' tiles of this stage
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), CG * C::STAGE_BYTES);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), CG * stage_tx);
           tma_load_2d_pair(sa, &tma_a, full_leader, kb * BK, m0);
-          tma_load_2d_pair(sb, &tma_b, full_leader, kb * BK, n0);
+          tma_load_2d_pair(sb, narrow ? &tma_bh : &tma_b, full_leader, kb * BK, n0);
           if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -240,8 +247,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
     // ------------------------------------------------------------------ MMA issuer (leader CTA only)
     if (lane == 0 && rank == 0) {
       // instruction descriptor: D fp32 (bit 4), A and B bf16 (bits 7, 10), both K-major, N >> 3 at 17, M >> 4 at 24
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
-                             ((uint32_t)((BM * CG) >> 4) << 24);
+      const uint32_t idesc0 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((BM * CG) >> 4) << 24);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -251,6 +257,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        const bool narrow = BN == 256 && g.N - (tile % tiles_n) * BN <= 128;
+        const uint32_t idesc = idesc0 | ((uint32_t)((narrow ? 128 : BN) >> 3) << 17);
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           fence_after();
@@ -431,7 +439,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
 }
 
 template <int BN, int EPI>
-cudaError_t launch_one(const TmaDesc& da, const TmaDesc& dw, const TmaDesc& dc, const GemmArgs& g, cudaStream_t s) {
+cudaError_t launch_one(const TmaDesc& da, const WeightDesc& dw, const TmaDesc& dc, const GemmArgs& g, cudaStream_t s) {
   using C = Cfg<BN>;
   static int max_pairs = 0;           // CTA pairs that can be resident at once (one CTA per SM)
   if (max_pairs == 0) {
@@ -465,11 +473,12 @@ cudaError_t launch_one(const TmaDesc& da, const TmaDesc& dw, const TmaDesc& dc, 
   cfg.attrs = attr; cfg.numAttrs = 1;
   ET_COUNT_LAUNCH();
   return cudaLaunchKernelEx(&cfg, gemm_bf16_kernel<BN, EPI>, *reinterpret_cast<const CUtensorMap*>(da.bytes),
-                            *reinterpret_cast<const CUtensorMap*>(dw.bytes), *reinterpret_cast<const CUtensorMap*>(dc.bytes), g);
+                            *reinterpret_cast<const CUtensorMap*>(dw.full.bytes), *reinterpret_cast<const CUtensorMap*>(dw.half.bytes),
+                            *reinterpret_cast<const CUtensorMap*>(dc.bytes), g);
 }
 
 template <int BN>
-cudaError_t launch_bn(const TmaDesc& da, const TmaDesc& dw, const TmaDesc& dc, const GemmArgs& g, int epilogue, cudaStream_t s) {
+cudaError_t launch_bn(const TmaDesc& da, const WeightDesc& dw, const TmaDesc& dc, const GemmArgs& g, int epilogue, cudaStream_t s) {
   switch (epilogue) {
     case EPI_STORE: return launch_one<BN, EPI_STORE>(da, dw, dc, g, s);
     case EPI_GELU: return launch_one<BN, EPI_GELU>(da, dw, dc, g, s);
@@ -521,6 +530,11 @@ bool make_tma_2d_bf16(TmaDesc* out, const void* base, uint64_t rows, uint64_t co
   return encode_2d(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, BK, box_rows, CU_TENSOR_MAP_SWIZZLE_128B, err);
 }
 
+bool make_tma_weight(WeightDesc* out, const void* base, uint64_t n_rows, uint64_t k_cols, const char** err) {
+  return make_tma_2d_bf16(&out->full, base, n_rows, k_cols, (uint32_t)gemm_bf16_w_box_rows((int)n_rows), err) &&
+         make_tma_2d_bf16(&out->half, base, n_rows, k_cols, 64, err);
+}
+
 bool make_tma_out(TmaDesc* out, const void* base, uint64_t rows, uint64_t cols, bool fp32, const char** err) {
   if (fp32) return encode_2d(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, rows, cols, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B, err);
   return encode_2d(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, rows, cols, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B, err);
@@ -535,7 +549,7 @@ int gemm_bf16_pick_bn(int N) {
 
 int gemm_bf16_w_box_rows(int N) { return gemm_bf16_pick_bn(N) / CG; }
 
-cudaError_t launch_gemm_bf16(const TmaDesc& da, const TmaDesc& dw, const TmaDesc& dc, const float* bias, void* c, int M_cap,
+cudaError_t launch_gemm_bf16(const TmaDesc& da, const WeightDesc& dw, const TmaDesc& dc, const float* bias, void* c, int M_cap,
                              int N, int K, int epilogue, int gelu_tanh, const float* table, int table_rows,
                              const int* n_frames_dev, int rows_per_frame, int* status_dev, cudaStream_t s) {
   GemmArgs g;
