@@ -176,7 +176,8 @@ def gelu_ref(x, tanh):
 
 @pytest.mark.parametrize("M,N,K", [(300, 1152, 1152), (257, 4304, 1152), (200, 3456, 1152), (333, 1152, 4304),
                                     (130, 1152, 592), (1, 256, 64), (128, 128, 128), (1000, 512, 72),
-                                    (2100, 4304, 1152), (1555, 3456, 256), (40000, 192, 64)])
+                                    (2100, 4304, 1152), (1555, 3456, 256), (40000, 192, 64),
+                                    (300, 72, 64), (513, 1160, 200), (256, 384, 1152), (777, 264, 8)])
 @pytest.mark.parametrize("epi", [0, 1, 2, 3])
 def test_linear_bf16(B, M, N, K, epi):
     import torch
