@@ -250,7 +250,9 @@ def test_attention_f32(B, n, L, H, dh):
 
 
 @pytest.mark.parametrize("n,L,H,dh", [(2, 729, 16, 72), (1, 64, 4, 16), (1, 100, 2, 64), (3, 130, 2, 72),
-                                      (1, 17, 1, 32), (1, 200, 1, 128), (1, 70, 2, 40)])
+                                      (1, 17, 1, 32), (1, 200, 1, 128), (1, 70, 2, 40),
+                                      (2, 128, 1, 72), (1, 257, 2, 72), (3, 1, 1, 72), (5, 16, 3, 64), (1, 513, 1, 72),
+                                      (40, 729, 2, 72)])
 def test_attention_bf16(B, n, L, H, dh):
     import torch
     rng = np.random.default_rng(L + dh)
