@@ -106,6 +106,10 @@ void launch_attention_scores_f32(const float* qkv, const float* lse, float* part
 void launch_attention_scores_bf16(const bf16* qkv, const float* lse, float* partial, float* score, int n_cap, int L,
                                   int heads, int dh, const int* n_frames_dev, cudaStream_t s);
 
+// scores_tcgen05.cu: the score pass on tcgen05 (head dims 64 and 72), same maps as the attention kernel
+cudaError_t launch_attention_scores_tc(const AttnMaps& maps, const float* lse, float* partial, float* score, int n_cap,
+                                       int L, int heads, int dh, const int* n_frames_dev, int* status_dev, cudaStream_t s);
+
 // ---- stage1.cu -----------------------------------------------------------------------------
 void launch_token_cosines(const float* x, float* cos_scratch, int n_cap, int L, int D, const int* n_frames_dev,
                           cudaStream_t s);

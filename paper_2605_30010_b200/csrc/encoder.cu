@@ -307,7 +307,8 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     });
     if (layer == c.num_layers - 1) {
       PROF(ET_CAT_SCORES, {
-        if (e->bf) launch_attention_scores_bf16((const bf16*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
+        if (e->attn_tc) ET_CUDA(e, launch_attention_scores_tc(e->attn_maps, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, e->d_small + 10, s));
+        else if (e->bf) launch_attention_scores_bf16((const bf16*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
         else launch_attention_scores_f32((const float*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
       });
     }
@@ -789,6 +790,12 @@ et_status et_attention_scores(const void* qkv_dev, const float* lse_dev, float* 
   cudaStream_t s = (cudaStream_t)cuda_stream;
   if (dtype == ET_BF16) {
     if (head_dim % 8 != 0) return ET_ERR_SHAPE;
+    if (attention_tc_supported(head_dim)) {
+      AttnMaps maps;
+      if (!make_attention_maps(&maps, (const bf16*)qkv_dev, (long long)n * L, heads, head_dim)) return ET_ERR_CUDA;
+      ET_CUDA0(launch_attention_scores_tc(maps, lse_dev, partial_dev, score_dev, n, L, heads, head_dim, nullptr, nullptr, s));
+      return ET_OK;
+    }
     launch_attention_scores_bf16((const bf16*)qkv_dev, lse_dev, partial_dev, score_dev, n, L, heads, head_dim, nullptr, s);
   } else if (dtype == ET_F32) {
     launch_attention_scores_f32((const float*)qkv_dev, lse_dev, partial_dev, score_dev, n, L, heads, head_dim, nullptr, s);
