@@ -140,6 +140,46 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
+def run_sweep(args, wl, enc, dev_vids, offs, n_rot, stream, barrier, torch):
+    """Timing columns in the shape of the paper's ablation tables (merge start layer, retained ratio, sampling
+    strategy, one stage only), on synthetic input: what changes is the work, not the accuracy."""
+    from dataclasses import replace
+    base = wl.params
+    T = wl.total_frames
+    settings = [("main setting", base), ("uncompressed", wl.uncompressed().params)]
+    for start in (4, 6, 8, 10):
+        settings.append((f"merge layers [{start},14,20]", replace(base, merge_layers=(start, 14, 20))))
+    for layers in ((10, 21, 23), (8, 21, 23)):
+        settings.append((f"merge layers {list(layers)}", replace(base, merge_layers=layers)))
+    for r in (0.25, 0.20, 0.15, 0.10):
+        settings.append((f"retain {r:.2f}", replace(base, retain=r)))
+    for tau in (0.5, 0.7, 0.9):
+        settings.append((f"tau_seg = tau_merge = {tau}", replace(base, tau_seg=tau, tau_merge=tau)))
+    settings += [("plain per-frame top-k", replace(base, selection=2)), ("random sampling", replace(base, selection=3, sample_seed=1)),
+                 ("unweighted merge", replace(base, weighted_merge=0)), ("stage I only", replace(base, selection=0)),
+                 ("stage II only", replace(base, merge_layers=()))]
+    steps = max(3, args.steps // 4)
+    ref_ms = None
+    for name, p in settings:
+        for i in range(2):
+            res = enc.encode_batch(dev_vids[i % n_rot], offs, p)
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for i in range(steps):
+            res = enc.encode_batch(dev_vids[i % n_rot], offs, p)
+        ev1.record(stream)
+        barrier()
+        ms = ev0.elapsed_time(ev1) / steps
+        if name == "uncompressed":
+            ref_ms = ms
+        print(json.dumps({"setting": name, "ms_per_call": round(ms, 3), "frames_per_s": round(T / (ms * 1e-3), 1),
+                          "frames_out": res.n_frames_out, "tokens_out": res.n_tokens,
+                          "tokens_kept": round(res.n_tokens / (T * wl.shape.tokens_per_frame), 4),
+                          "frames_per_block": res.frames_per_block,
+                          "speedup_vs_uncompressed": round(ref_ms / ms, 3) if ref_ms else None}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -148,6 +188,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="so400m_32f")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the benchmark line, time the paper's ablation settings (merge start layer, retained "
+                         "ratio, sampling strategy, single stages) on the workload and print one JSON line per setting")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -221,6 +264,13 @@ def main():
     barrier()
     prof = B.et_profile_read(enc)
     B.et_profile_enable(enc, False)
+
+    if args.sweep:
+        if rank == 0:
+            run_sweep(args, wl, enc, dev_vids, offs, n_rot, stream, barrier, torch)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
 
     # ---------------- end to end through the host entry point (pinned host frames in, host tokens out)
     dst = B.HostBuffers(T * shape.tokens_per_frame, T, shape.hidden, V)
