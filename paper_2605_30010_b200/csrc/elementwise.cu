@@ -9,6 +9,9 @@ namespace et {
 // Patch feature index = c*p*p + dy*p + dx, i.e. the flattening of a [D][3][p][p] convolution
 // weight; columns >= 3*p*p are zero (pad so that the row pitch is a multiple of 16 bytes).
 // ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void store_pair(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store_pair(bf16* p, float a, float b) { *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b); }
+
 template <typename T>
 __global__ void im2col_kernel(const float* __restrict__ frames, T* __restrict__ patches, int T_frames, int image,
                               int patch, int grid, int k_pad, const int* __restrict__ n_frames_dev) {
@@ -30,7 +33,16 @@ __global__ void im2col_kernel(const float* __restrict__ frames, T* __restrict__ 
     const int gy = l / grid, gx = l % grid;
     const float* src = frames + (((long long)f * 3 + c) * image + (gy * patch + dy)) * image + gx * patch;
     T* dst = dst_row + (c * patch + dy) * patch;
-    for (int dx = 0; dx < patch; ++dx) dst[dx] = to_out<T>(__ldg(src + dx));
+    if ((patch & 1) == 0 && (image & 1) == 0 && (k_pad & 1) == 0 && (reinterpret_cast<size_t>(frames) & 7) == 0) {
+      // pixel pairs: the patch row starts at an even pixel of an even-width image and at an even patch column
+      const float2* s2 = reinterpret_cast<const float2*>(src);
+      for (int dx = 0; dx < patch; dx += 2) {
+        const float2 v = __ldg(s2 + (dx >> 1));
+        store_pair(dst + dx, v.x, v.y);
+      }
+    } else {
+      for (int dx = 0; dx < patch; ++dx) dst[dx] = to_out<T>(__ldg(src + dx));
+    }
   }
 }
 
