@@ -558,7 +558,6 @@ cudaError_t launch_gemm_bf16(const TmaDesc& da, const WeightDesc& dw, const TmaD
   g.n_frames_dev = n_frames_dev; g.rows_per_frame = rows_per_frame; g.status = status_dev;
   switch (gemm_bf16_pick_bn(N)) {
     case 256: return launch_bn<256>(da, dw, dc, g, epilogue, s);
-    case 192: return launch_bn<192>(da, dw, dc, g, epilogue, s);
     default: return launch_bn<128>(da, dw, dc, g, epilogue, s);
   }
 }
