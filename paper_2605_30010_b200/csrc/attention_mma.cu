@@ -95,7 +95,7 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, float
   const bf16* vg = qg + 2 * D;
 
   // zero the padded contraction columns [DH, DHP) of Q and K once (cp.async never writes them)
-  if (G::DHP > DH) {
+  if constexpr (G::DHP > DH) {
     constexpr int PADC = G::DHP - DH;
     for (int i = tid; i < (QT + 2 * KT) * PADC; i += 128) {
       const int r = i / PADC, c = DH + i % PADC;
@@ -256,7 +256,7 @@ score_mma_kernel(const bf16* __restrict__ qkv, const float* __restrict__ lse, fl
   const bf16* qg = qkv + (size_t)f * L * row_stride + (size_t)h * DH;
   const bf16* kg = qg + D;
   const float* lse_row = lse + ((size_t)f * heads + h) * L;
-  if (G::DHP > DH) {
+  if constexpr (G::DHP > DH) {
     constexpr int PADC = G::DHP - DH;
     for (int i = tid; i < (KT + 2 * QT) * PADC; i += 128) {
       const int r = i / PADC, c = DH + i % PADC;

@@ -12,7 +12,6 @@ template <> __device__ __forceinline__ float ld_f<bf16>(const bf16* p) { return 
 
 constexpr int AS_QB = 16;     // queries per CTA (4 per warp)
 constexpr int AS_KC = 32;     // keys per chunk (one per lane)
-constexpr int AS_MAX_DH = 128;
 
 // grid (ceil(L/AS_QB), heads, frames), 128 threads.  qkv [n*L][3*D] with D = heads*dh.
 template <typename T>

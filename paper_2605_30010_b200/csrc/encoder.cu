@@ -481,7 +481,6 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
     return bail(ET_ERR_CUDA);
   const size_t es = e->bf ? 2 : 4;
   // ---- activations
-  void* tmp = nullptr;
 #define ET_A(ptr, bytes)                                                     \
   do {                                                                       \
     unsigned char* q__ = nullptr;                                            \
@@ -508,7 +507,6 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   ET_A(e->frame_offsets, (F + 1) * 4); ET_A(e->token_pos, rows * 4); ET_A(e->tokens, rows * D * 4);
   ET_A(e->d_small, 16 * 4);
 #undef ET_A
-  (void)tmp;
   if ((st = halloc(e, &e->h_small, 16)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_vid_off, e->Vmax + 1)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_forced, 2 * ET_MAX_MERGE_LAYERS * F)) != ET_OK) return bail(st);

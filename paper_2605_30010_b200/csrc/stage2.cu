@@ -215,7 +215,6 @@ void launch_scan_counts(const int* count, int* frame_offsets, int* totals, int n
 // per step, carry in a register), then its warps move their share of the kept rows:
 // warp-per-row, row in registers, LayerNorm statistics by shuffles.
 // ---------------------------------------------------------------------------------------------
-constexpr int GATHER_MAX_L = 4096;
 
 template <int NV>
 __global__ void __launch_bounds__(256)
