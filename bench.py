@@ -62,6 +62,12 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
+    def wait_first_sample(self, timeout_s: float):
+        """Blocks until nvidia-smi has printed once: its start-up (driver queries) is over by then."""
+        t0 = time.time()
+        while self.proc is not None and not self.lines and time.time() - t0 < timeout_s:
+            time.sleep(0.05)
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -243,6 +249,7 @@ def main():
     # ---------------- device-resident timing (the headline `value`), no per-kernel events in the stream
     sampler = ClockSampler(local)
     sampler.start()                              # started before the warm-up: its start-up cost stays out of the timed steps
+    sampler.wait_first_sample(3.0)
     for i in range(args.warmup):
         res = enc.encode_batch(dev_vids[i % n_rot], offs, params)
     barrier()
