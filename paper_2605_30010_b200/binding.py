@@ -23,7 +23,10 @@ EXPORTS = ["et_encoder_create", "et_encode_video", "et_encode_batch", "et_encode
            "et_status_string", "et_last_error", "et_kernel_launch_count", "et_profile_enable", "et_profile_read",
            "et_frame_similarity_static", "et_frame_similarity", "et_merge_plan",
            "et_merge_frames", "et_select_tokens", "et_gather_tokens", "et_linear_bf16", "et_attention",
-           "et_attention_scores", "et_layernorm"]
+           "et_attention_scores", "et_layernorm",
+           # include/earlytom_llm.h
+           "et_llm_create", "et_llm_prefill", "et_llm_destroy", "et_llm_last_error", "et_llm_profile_enable",
+           "et_llm_profile_read", "et_rmsnorm", "et_rope", "et_swiglu", "et_attention_causal"]
 
 
 class EarlyTomError(RuntimeError):
@@ -91,6 +94,28 @@ class et_profile(C.Structure):
                 ("launches", C.c_ulonglong * ET_PROF_CATS), ("calls", C.c_int)]
 
 
+class et_llm_config(C.Structure):
+    _fields_ = [("vision_hidden", C.c_int), ("hidden", C.c_int), ("num_layers", C.c_int), ("heads", C.c_int),
+                ("kv_heads", C.c_int), ("head_dim", C.c_int), ("mlp_dim", C.c_int), ("vocab", C.c_int),
+                ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("gelu_tanh", C.c_int), ("max_tokens", C.c_int)]
+
+
+class et_llm_weights(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("count", C.c_size_t), ("on_device", C.c_int)]
+
+
+class et_llm_result(C.Structure):
+    _fields_ = [("n_tokens", C.c_int), ("first_token", C.c_int), ("logits", C.c_void_p), ("hidden", C.c_void_p)]
+
+
+ET_LLM_CATS = 8
+LLM_PROF_NAMES = ["embed", "norm", "gemm", "rope", "attention", "swiglu", "head"]
+
+
+class et_llm_profile(C.Structure):
+    _fields_ = [("ms", C.c_double * ET_LLM_CATS), ("launches", C.c_ulonglong * ET_LLM_CATS), ("calls", C.c_int)]
+
+
 def load_library(path: str = _LIB_PATH) -> C.CDLL:
     if not os.path.exists(path):
         raise ImportError(f"{path} is missing: build it with `python -m paper_2605_30010_b200.build` "
@@ -124,10 +149,22 @@ def load_library(path: str = _LIB_PATH) -> C.CDLL:
     lib.et_attention.argtypes = [vp, vp, vp, i, i, i, i, i, vp]
     lib.et_attention_scores.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp]
     lib.et_layernorm.argtypes = [vp, vp, vp, f, vp, i, i, i, vp]
+    lib.et_llm_create.argtypes = [C.POINTER(et_llm_config), C.POINTER(et_llm_weights), C.POINTER(vp)]
+    lib.et_llm_prefill.argtypes = [vp, _I32P, i, vp, i, _I32P, i, vp, C.POINTER(et_llm_result)]
+    lib.et_llm_destroy.argtypes = [vp]
+    lib.et_llm_destroy.restype = None
+    lib.et_llm_last_error.argtypes = [vp]
+    lib.et_llm_last_error.restype = C.c_char_p
+    lib.et_llm_profile_enable.argtypes = [vp, i]
+    lib.et_llm_profile_read.argtypes = [vp, C.POINTER(et_llm_profile)]
+    lib.et_rmsnorm.argtypes = [vp, vp, f, vp, i, i, vp]
+    lib.et_rope.argtypes = [vp, i, i, i, i, i, f, vp]
+    lib.et_swiglu.argtypes = [vp, vp, i, i, vp]
+    lib.et_attention_causal.argtypes = [vp, vp, i, i, i, i, i, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name.startswith("et_") and name not in ("et_destroy", "et_status_string", "et_last_error",
-                                                  "et_kernel_launch_count"):
+                                                  "et_kernel_launch_count", "et_llm_destroy", "et_llm_last_error"):
             fn.restype = C.c_int
     return lib
 
@@ -516,3 +553,125 @@ def et_layernorm(x, g, b, eps, out_bf16=False, stream=None):
     _check(lib().et_layernorm(_ptr(x), _ptr(g), _ptr(b), float(eps), _ptr(y), rows, D, ET_BF16 if out_bf16 else ET_F32,
                               _stream_ptr(stream)))
     return y
+
+
+# --------------------------------------------------------------------------------------------
+# Downstream of the encoder: projector + language-model prefill (include/earlytom_llm.h)
+# --------------------------------------------------------------------------------------------
+
+@dataclass
+class PrefillResult:
+    n_tokens: int
+    first_token: int
+    logits: object        # torch fp32 [vocab] (copy)
+    hidden: object        # torch fp32 [n_tokens, hidden] (copy) or None
+
+
+def et_llm_create(cfg: et_llm_config, weights) -> C.c_void_p:
+    """weights: numpy fp32 blob (host) or a torch fp32 CUDA tensor (device blob)."""
+    if isinstance(weights, np.ndarray):
+        w = np.ascontiguousarray(weights, dtype=np.float32)
+        wb = et_llm_weights(w.ctypes.data, w.size, 0)
+    else:
+        assert weights.is_cuda and weights.is_contiguous() and weights.element_size() == 4
+        wb = et_llm_weights(weights.data_ptr(), weights.numel(), 1)
+    h = C.c_void_p()
+    _check(lib().et_llm_create(C.byref(cfg), C.byref(wb), C.byref(h)))
+    return h
+
+
+def et_llm_destroy(handle) -> None:
+    lib().et_llm_destroy(handle)
+
+
+class LanguageModel:
+    """Owns an et_llm*.  `shape` is any object with the architecture fields of et_llm_config."""
+
+    def __init__(self, shape, weights, max_tokens: int):
+        cfg = et_llm_config(shape.vision_hidden, shape.hidden, shape.num_layers, shape.heads, shape.kv_heads, shape.head_dim,
+                            shape.mlp_dim, shape.vocab, float(shape.rms_eps), float(shape.rope_theta), int(shape.gelu_tanh),
+                            int(max_tokens))
+        self.handle = et_llm_create(cfg, weights)
+        self.shape = shape
+
+    def close(self):
+        if getattr(self, "handle", None):
+            et_llm_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def prefill(self, prefix_ids, visual_tokens, suffix_ids, want_hidden=False, stream=None) -> PrefillResult:
+        return et_llm_prefill(self, prefix_ids, visual_tokens, suffix_ids, want_hidden, stream)
+
+
+def _ids(a):
+    a = np.ascontiguousarray(a if a is not None else [], dtype=np.int32)
+    return a, (a.ctypes.data_as(_I32P) if a.size else None)
+
+
+def et_llm_prefill(llm: LanguageModel, prefix_ids, visual_tokens, suffix_ids, want_hidden=False, stream=None,
+                   copy_logits=True) -> PrefillResult:
+    """visual_tokens: torch fp32 CUDA [n_visual, vision_hidden] (or None)."""
+    pre, pre_p = _ids(prefix_ids)
+    suf, suf_p = _ids(suffix_ids)
+    n_vis = 0
+    if visual_tokens is not None and visual_tokens.shape[0] > 0:
+        assert visual_tokens.is_cuda and visual_tokens.is_contiguous() and visual_tokens.element_size() == 4
+        assert visual_tokens.shape[1] == llm.shape.vision_hidden
+        n_vis = int(visual_tokens.shape[0])
+    r = et_llm_result()
+    st = lib().et_llm_prefill(llm.handle, pre_p, int(pre.size), _ptr(visual_tokens) if n_vis else None, n_vis, suf_p,
+                              int(suf.size), _stream_ptr(stream), C.byref(r))
+    if st != 0:
+        raise EarlyTomError(st, lib().et_llm_last_error(llm.handle).decode())
+    logits = _dev_tensor(r.logits, (llm.shape.vocab,), "<f4") if copy_logits else None
+    hidden = _dev_tensor(r.hidden, (r.n_tokens, llm.shape.hidden), "<f4") if want_hidden else None
+    return PrefillResult(r.n_tokens, r.first_token, logits, hidden)
+
+
+def et_llm_profile_enable(llm: LanguageModel, on: bool) -> None:
+    _check(lib().et_llm_profile_enable(llm.handle, 1 if on else 0))
+
+
+def et_llm_profile_read(llm: LanguageModel) -> dict:
+    p = et_llm_profile()
+    _check(lib().et_llm_profile_read(llm.handle, C.byref(p)))
+    return {"calls": p.calls, "ms": {n: p.ms[k] for k, n in enumerate(LLM_PROF_NAMES)},
+            "launches": {n: int(p.launches[k]) for k, n in enumerate(LLM_PROF_NAMES)}}
+
+
+def et_rmsnorm(x, g, eps, stream=None):
+    import torch
+    rows, D = x.shape
+    y = torch.empty((rows, D), dtype=torch.bfloat16, device=x.device)
+    _check(lib().et_rmsnorm(_ptr(x), _ptr(g), float(eps), _ptr(y), rows, D, _stream_ptr(stream)))
+    return y
+
+
+def et_rope(qkv, L, heads, kv_heads, head_dim, theta, stream=None):
+    """In place on qkv (bf16 [rows, (heads + 2*kv_heads)*head_dim]); returns qkv."""
+    _check(lib().et_rope(_ptr(qkv), int(qkv.shape[0]), int(L), heads, kv_heads, head_dim, float(theta), _stream_ptr(stream)))
+    return qkv
+
+
+def et_swiglu(gu, stream=None):
+    import torch
+    rows, M2 = gu.shape
+    h = torch.empty((rows, M2 // 2), dtype=torch.bfloat16, device=gu.device)
+    _check(lib().et_swiglu(_ptr(gu), _ptr(h), rows, M2 // 2, _stream_ptr(stream)))
+    return h
+
+
+def et_attention_causal(qkv, n_seq, L, heads, kv_heads, head_dim, stream=None):
+    """Returns (out bf16 [n_seq*L, heads*head_dim], status int32[1])."""
+    import torch
+    out = torch.empty((n_seq * L, heads * head_dim), dtype=torch.bfloat16, device=qkv.device)
+    status = torch.zeros(1, dtype=torch.int32, device=qkv.device)
+    _check(lib().et_attention_causal(_ptr(qkv), _ptr(out), n_seq, L, heads, kv_heads, head_dim, _ptr(status),
+                                     _stream_ptr(stream)))
+    return out, status

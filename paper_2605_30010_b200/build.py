@@ -31,7 +31,8 @@ def sources():
 
 def _deps_mtime():
     files = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
-    files.append(os.path.join(ROOT, "include", "earlytom.h"))
+    inc = os.path.join(ROOT, "include")
+    files += [os.path.join(inc, f) for f in os.listdir(inc) if f.endswith(".h")]
     return max(os.path.getmtime(f) for f in files)
 
 

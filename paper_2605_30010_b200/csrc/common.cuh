@@ -110,6 +110,27 @@ void launch_attention_scores_bf16(const bf16* qkv, const float* lse, float* part
 cudaError_t launch_attention_scores_tc(const AttnMaps& maps, const float* lse, float* partial, float* score, int n_cap,
                                        int L, int heads, int dh, const int* n_frames_dev, int* status_dev, cudaStream_t s);
 
+// attention_causal_tcgen05.cu: causal grouped-query attention, head dim 128, over packed rows
+// [heads*128 | kv_heads*128 | kv_heads*128] of n_seq sequences of L positions each.
+bool attention_causal_supported(int head_dim);
+bool make_causal_attention_map(TmaDesc* out, const bf16* qkv, long long rows, int heads, int kv_heads);
+cudaError_t launch_attention_causal(const TmaDesc& map, bf16* out, int n_seq, int L, int heads, int kv_heads,
+                                    int* status_dev, cudaStream_t s);
+
+// ---- llm_ops.cu: row-wise and elementwise steps of the language model --------------------------
+// y = x * rsqrt(mean(x^2) + eps) * g, rows [rows][D] fp32 -> bf16
+void launch_rmsnorm(const float* x, const float* g, float eps, bf16* y, int rows, int D, cudaStream_t s);
+// rotate-half rotary embedding in place on the Q and K parts of packed rows [rows][(heads + 2*kv_heads)*dh];
+// the position of a row is row % L; inv_turns [dh/2] (device, double) = theta^(-2i/dh) / (2 pi)
+void launch_rope(bf16* qkv, int rows, int L, int heads, int kv_heads, int dh, const double* inv_turns, cudaStream_t s);
+// h[r][j] = silu(gu[r][j]) * gu[r][M + j]
+void launch_swiglu(const bf16* gu, bf16* h, int rows, int M, cudaStream_t s);
+// x[r][:] = table[ids[r]][:]  (bf16 table -> fp32 rows)
+void launch_embed_rows(const bf16* table, const int* ids, float* x, int rows, int D, int vocab, cudaStream_t s);
+void launch_cast_bf16(const float* x, bf16* y, size_t count, cudaStream_t s);
+// first index of the maximum of x[0..n)
+void launch_argmax(const float* x, int n, int* out, cudaStream_t s);
+
 // ---- stage1.cu -----------------------------------------------------------------------------
 void launch_token_cosines(const float* x, float* cos_scratch, int n_cap, int L, int D, const int* n_frames_dev,
                           cudaStream_t s);

@@ -6,11 +6,11 @@ import re
 import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-HEADER = os.path.join(ROOT, "include", "earlytom.h")
+HEADERS = [os.path.join(ROOT, "include", f) for f in sorted(os.listdir(os.path.join(ROOT, "include"))) if f.endswith(".h")]
 
 
 def declared_symbols():
-    text = open(HEADER).read()
+    text = "".join(open(h).read() for h in HEADERS)
     return sorted(set(re.findall(r"ET_API[^;(]*?\b(et_[a-z0-9_]+)\s*\(", text)))
 
 
@@ -30,14 +30,14 @@ def test_header_declares_the_boundary_calls():
 def test_library_exports_every_declared_symbol(built_lib):
     lib = ctypes.CDLL(built_lib)
     for s in declared_symbols():
-        assert hasattr(lib, s), f"{s} is declared in earlytom.h but not exported"
+        assert hasattr(lib, s), f"{s} is declared in include/*.h but not exported"
 
 
 def test_binding_covers_every_declared_symbol(built_lib):
     from paper_2605_30010_b200 import binding
     assert sorted(binding.EXPORTS) == declared_symbols()
     for s in declared_symbols():
-        assert hasattr(binding, s) or s in ("et_status_string", "et_last_error"), s
+        assert hasattr(binding, s) or s in ("et_status_string", "et_last_error", "et_llm_last_error"), s
 
 
 def test_struct_sizes_match_the_header(built_lib, tmp_path):
@@ -45,14 +45,16 @@ def test_struct_sizes_match_the_header(built_lib, tmp_path):
     import subprocess
     from paper_2605_30010_b200 import binding as b
     src = tmp_path / "sz.c"
-    src.write_text('#include <stdio.h>\n#include "earlytom.h"\nint main(){printf("%zu %zu %zu %zu %zu %zu %zu\\n",'
+    src.write_text('#include <stdio.h>\n#include "earlytom_llm.h"\nint main(){printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu %zu %zu\\n",'
                    'sizeof(et_config),sizeof(et_weights),sizeof(et_forced_plan),sizeof(et_params),sizeof(et_trace),'
-                   'sizeof(et_result),sizeof(et_host_buffers));return 0;}\n')
+                   'sizeof(et_result),sizeof(et_host_buffers),sizeof(et_llm_config),sizeof(et_llm_weights),'
+                   'sizeof(et_llm_result),sizeof(et_llm_profile));return 0;}\n')
     exe = tmp_path / "sz"
     subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     sizes = [int(x) for x in subprocess.check_output([str(exe)]).split()]
     mine = [ctypes.sizeof(t) for t in (b.et_config, b.et_weights, b.et_forced_plan, b.et_params, b.et_trace,
-                                       b.et_result, b.et_host_buffers)]
+                                       b.et_result, b.et_host_buffers, b.et_llm_config, b.et_llm_weights,
+                                       b.et_llm_result, b.et_llm_profile)]
     assert sizes == mine
 
 
