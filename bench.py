@@ -186,6 +186,68 @@ def run_sweep(args, wl, enc, dev_vids, offs, n_rot, stream, barrier, torch):
                           "speedup_vs_uncompressed": round(ref_ms / ms, 3) if ref_ms else None}))
 
 
+def run_downstream(args, wl, enc, dev_vids, offs, stream, peaks, torch, B):
+    """Time-to-first-token in the manner of the paper's Fig. 1: encoder call, then projector + language-model prefill of
+    [text | visual tokens | text] up to the first token, chained on the device.  Qwen2-7B shapes (the language model of
+    LLaVA-OneVision-7B) with random-init weights drawn on the device; three settings of the encoder."""
+    from dataclasses import replace
+    from synthetic.llm import QWEN2_7B, make_llm_weights_device, make_prompt
+    shape = QWEN2_7B
+    T, L = wl.total_frames, wl.shape.tokens_per_frame
+    n_text = (14, 40)
+    blob = make_llm_weights_device(shape, 77)
+    llm = B.LanguageModel(shape, blob, max_tokens=T * L + sum(n_text))
+    del blob
+    torch.cuda.empty_cache()
+    pre, suf = make_prompt(shape, n_text[0], n_text[1], 77)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    settings = [("main setting (retain 0.25)", wl.params), ("retain 0.10", replace(wl.params, retain=0.10)),
+                ("uncompressed encoder, all tokens", wl.uncompressed().params)]
+    rows, prof_main = [], None
+    steps = 5
+    try:
+        for name, p in settings:
+            for i in range(2):
+                res = enc.encode_batch(dev_vids[i % len(dev_vids)], offs, p)
+                B.et_llm_prefill(llm, pre, res.tokens, suf, copy_logits=False)
+            torch.cuda.synchronize()
+            enc_ms = llm_ms = 0.0
+            for i in range(steps):
+                ev[0].record(stream)
+                res = enc.encode_batch(dev_vids[i % len(dev_vids)], offs, p)
+                ev[1].record(stream)
+                out = B.et_llm_prefill(llm, pre, res.tokens, suf, copy_logits=False)
+                ev[2].record(stream)
+                torch.cuda.synchronize()
+                enc_ms += ev[0].elapsed_time(ev[1]) / steps
+                llm_ms += ev[1].elapsed_time(ev[2]) / steps
+            rows.append({"setting": name, "visual_tokens": res.n_tokens, "sequence": out.n_tokens, "encoder_ms": round(enc_ms, 3),
+                         "projector_prefill_ms": round(llm_ms, 3), "ttft_ms": round(enc_ms + llm_ms, 3)})
+            if prof_main is None:
+                B.et_llm_profile_enable(llm, True)
+                for i in range(3):
+                    B.et_llm_prefill(llm, pre, res.tokens, suf, copy_logits=False)
+                prof_main = B.et_llm_profile_read(llm)
+                B.et_llm_profile_enable(llm, False)
+                n, n_vis = out.n_tokens, res.n_tokens
+    finally:
+        llm.close()
+    H, M = shape.hidden, shape.mlp_dim
+    gemm_flops = shape.num_layers * 2.0 * n * (H * shape.qkv_dim + shape.q_dim * H + 3 * H * M) \
+        + 2.0 * n_vis * (shape.vision_hidden * H + H * H) + 2.0 * H * shape.vocab
+    attn_flops = shape.num_layers * 2.0 * n * n * shape.q_dim              # causal: half of the n^2 products
+    calls = prof_main["calls"]
+    gemm_tf = gemm_flops / (prof_main["ms"]["gemm"] / calls * 1e-3) / 1e12
+    attn_tf = attn_flops / (prof_main["ms"]["attention"] / calls * 1e-3) / 1e12
+    return {"model": "Qwen2-7B shapes (28 layers, hidden 3584, 28 query / 4 key-value heads of 128, MLP 18944, vocab 152064), "
+                     "random init drawn on the device, bf16", "text_tokens": sum(n_text), "steps": steps, "settings": rows,
+            "ttft_speedup_vs_uncompressed": round(rows[-1]["ttft_ms"] / rows[0]["ttft_ms"], 3),
+            "prefill_main_setting": {"ms_per_stage": {k: round(v / calls, 3) for k, v in prof_main["ms"].items()},
+                                     "gemm_tflops": round(gemm_tf, 1), "gemm_frac_of_bf16_peak": round(gemm_tf / peaks["bf16_tflops_sustained"], 3),
+                                     "attention_tflops": round(attn_tf, 1),
+                                     "launches": sum(prof_main["launches"].values()) // calls}}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -194,6 +256,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="so400m_32f")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-downstream", action="store_true",
+                    help="skip the time-to-first-token figures (projector + 7B-shape language-model prefill after the encoder)")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark line, time the paper's ablation settings (merge start layer, retained "
                          "ratio, sampling strategy, single stages) on the workload and print one JSON line per setting")
@@ -350,6 +414,11 @@ def main():
                     "ms_per_step": e2e_ms_step},
             "uncompressed": {"ms_per_video": unc_ms, "frames_per_s": T / (unc_ms * 1e-3), "speedup_of_compression": unc_ms / ms_step},
             "roofline": roofline, "kernels": per_cat}
+    if not args.no_downstream and world == 1 and wl.name == "so400m_32f":
+        try:
+            line["downstream"] = run_downstream(args, wl, enc, dev_vids, offs, stream, peaks, torch, B)
+        except Exception as ex:          # the headline line never depends on this stage
+            line["downstream"] = {"error": f"{type(ex).__name__}: {ex}"}
     if not args.no_cpu_baseline:
         sample = 2
         fps, dt, cores = oracle_sample(wl, vids[0], blob, sample, 1, 1)
