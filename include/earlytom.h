@@ -274,7 +274,10 @@ ET_API et_status et_gather_tokens(const float* x_dev, const unsigned char* keep_
 /* Dense layer on the tensor cores (the GEMMs of the encoder blocks, paper Eq. 8's 4LD^2 + 2LDM
  * terms): c = epilogue(a[M][K] * w[N][K]^T + bias[N]).  a_dev, w_dev bf16 (K contiguous, K*2 bytes
  * a multiple of 16); epilogue 0: store bf16; 1: GELU then store bf16; 2: c fp32 += result
- * (residual, in place); 3: c fp32 = result + table[(row % table_rows)][N] (position embedding).
+ * (residual, in place); 3: c fp32 = result + table[(row % table_rows)][N] (position embedding);
+ * 4: gated feed-forward of the language model (earlytom_llm.h): the rows of w are ordered in tiles of
+ * 256 = four groups of (32 gate rows, 32 up rows) of the same 32 outputs, bias is ignored, N % 256 == 0 and
+ * c is bf16 [M][N/2] = silu(gate) * up.
  * status_dev int [1] receives a non-zero code if a bounded wait expired. */
 ET_API et_status et_linear_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, void* c_dev, int M, int N,
                          int K, int epilogue, int gelu_tanh, const float* table_dev, int table_rows,

@@ -519,7 +519,8 @@ def et_linear_bf16(a, w, bias, epilogue=0, gelu_tanh=1, c=None, table=None, stre
     M, K = a.shape
     N = w.shape[0]
     if c is None:
-        c = torch.empty((M, N), dtype=torch.bfloat16 if epilogue in (0, 1) else torch.float32, device=a.device)
+        c = torch.empty((M, N // 2 if epilogue == 4 else N), dtype=torch.bfloat16 if epilogue in (0, 1, 4) else torch.float32,
+                        device=a.device)
     status = torch.zeros(1, dtype=torch.int32, device=a.device)
     _check(lib().et_linear_bf16(_ptr(a), _ptr(w), _ptr(bias), _ptr(c), M, N, K, int(epilogue), int(gelu_tanh),
                                 _ptr(table), int(table.shape[0]) if table is not None else 0, _ptr(status),

@@ -51,7 +51,9 @@ struct LayerTrace {
   unsigned char* merge_next;
 };
 
-enum Epilogue : int { EPI_STORE = 0, EPI_GELU = 1, EPI_RESIDUAL = 2, EPI_TABLE = 3 };
+// EPI_SWIGLU: the N accumulator columns are pairs of 32-column chunks (gate, up) of the same 32 outputs; the layer
+// writes c [M][N/2] = silu(gate) * up in bf16 and takes no bias.  N % 256 == 0.
+enum Epilogue : int { EPI_STORE = 0, EPI_GELU = 1, EPI_RESIDUAL = 2, EPI_TABLE = 3, EPI_SWIGLU = 4 };
 
 // ---- elementwise.cu ------------------------------------------------------------------------
 // frames fp32 [T][3][H][W] -> patches [T*L][k_pad] (zero padded beyond 3*p*p), fp32 or bf16.

@@ -746,12 +746,13 @@ et_status et_linear_bf16(const void* a_dev, const void* w_dev, const float* bias
                          void* cuda_stream) {
   if (!a_dev || !w_dev || !bias_dev || !c_dev) return ET_ERR_INVALID_ARG;
   if (M < 1 || N < 8 || N % 8 != 0 || K < 8 || K % 8 != 0) return ET_ERR_SHAPE;
-  if (epilogue < 0 || epilogue > 3 || (epilogue == 3 && (!table_dev || table_rows < 1))) return ET_ERR_INVALID_ARG;
+  if (epilogue < 0 || epilogue > 4 || (epilogue == 3 && (!table_dev || table_rows < 1))) return ET_ERR_INVALID_ARG;
+  if (epilogue == 4 && N % 256 != 0) return ET_ERR_SHAPE;
   TmaDesc da, dc;
   WeightDesc dw;
   const char* err = nullptr;
   if (!make_tma_2d_bf16(&da, a_dev, M, K, 128, &err) || !make_tma_weight(&dw, w_dev, N, K, &err) ||
-      !make_tma_out(&dc, c_dev, M, N, epilogue >= 2, &err))
+      !make_tma_out(&dc, c_dev, M, epilogue == 4 ? N / 2 : N, epilogue == 2 || epilogue == 3, &err))
     return ET_ERR_CUDA;
   ET_CUDA0(launch_gemm_bf16(da, dw, dc, bias_dev, c_dev, M, N, K, epilogue, gelu_tanh, table_dev, table_rows, nullptr, 1,
                             status_dev, (cudaStream_t)cuda_stream));

@@ -303,6 +303,40 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
           uint32_t rr[2][32];
           const int c_first = half * CH_PER * 32;
           if (n0 + c_first < g.N) tmem_ld32_async(t_row + (uint32_t)c_first, rr[0]);
+          if constexpr (EPI == EPI_SWIGLU) {
+            // Chunks come in pairs (gate, up) of the same 32 outputs (the weight rows were interleaved that way):
+            // h = silu(gate) * up, half as many output columns as accumulator columns.  No bias.
+            float gate[32];
+#pragma unroll
+            for (int ch = 0; ch < CH_PER; ++ch) {
+              const int c0 = (half * CH_PER + ch) * 32;
+              tmem_wait_ld();
+              tmem_regs_ready(rr[ch & 1]);
+              if (ch + 1 < CH_PER) tmem_ld32_async(t_row + (uint32_t)(c0 + 32), rr[(ch + 1) & 1]);
+              const uint32_t (&r)[32] = rr[ch & 1];
+              if ((ch & 1) == 0) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) gate[i] = __uint_as_float(r[i]);
+              } else {
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __fdividef(gate[i], 1.f + __expf(-gate[i])) * __uint_as_float(r[i]);
+                if (lane == 0) bulk_wait_read<1>();   // the half written two stores ago has been read
+                __syncwarp();
+                const uint32_t buf = slab + sub * 2048u;
+                const uint32_t rowp = buf + (uint32_t)lane * 64u;
+                const uint32_t sw = (uint32_t)(lane >> 1) & 3u;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  st_shared_v4(rowp + ((((uint32_t)j) ^ sw) << 4), pack_bf16(v[j * 8 + 0], v[j * 8 + 1]), pack_bf16(v[j * 8 + 2], v[j * 8 + 3]),
+                               pack_bf16(v[j * 8 + 4], v[j * 8 + 5]), pack_bf16(v[j * 8 + 6], v[j * 8 + 7]));
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) { tma_store_2d(&tma_c, buf, (n0 + c0 - 32) >> 1, m0 + quarter * 32); bulk_commit(); }
+                sub ^= 1u;
+              }
+            }
+          } else {
 #pragma unroll
           for (int ch = 0; ch < CH_PER; ++ch) {
             const int c0 = (half * CH_PER + ch) * 32;
@@ -361,6 +395,33 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
               fence_async_smem();
               __syncwarp();
               if (lane == 0) { tma_reduce_add_2d(&tma_c, slab, col0, m0 + quarter * 32); bulk_commit(); }
+            }
+          }
+          }
+        } else if constexpr (EPI == EPI_SWIGLU) {
+          // ---- last row tile of the gated layer: per-row stores of silu(gate) * up, rows >= M untouched
+          const int row = m0 + quarter * 32 + lane;
+          const bool row_ok = row < M;
+#pragma unroll 1
+          for (int pr = 0; pr < CH_PER / 2; ++pr) {
+            const int c0 = (half * CH_PER + 2 * pr) * 32;
+            uint32_t rg[32], ru[32];
+            tmem_ld32(t_row + (uint32_t)c0, rg);
+            tmem_ld32(t_row + (uint32_t)(c0 + 32), ru);
+            if (!row_ok) continue;
+            bf16* dst = reinterpret_cast<bf16*>(g.c) + (size_t)row * (size_t)(g.N >> 1) + ((n0 + c0) >> 1);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              float v[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const float gt = __uint_as_float(rg[q * 8 + i]);
+                v[i] = __fdividef(gt, 1.f + __expf(-gt)) * __uint_as_float(ru[q * 8 + i]);
+              }
+              uint4 o;
+              o.x = pack_bf16(v[0], v[1]); o.y = pack_bf16(v[2], v[3]);
+              o.z = pack_bf16(v[4], v[5]); o.w = pack_bf16(v[6], v[7]);
+              *reinterpret_cast<uint4*>(dst + q * 8) = o;
             }
           }
         } else {
@@ -484,6 +545,10 @@ cudaError_t launch_bn(const TmaDesc& da, const WeightDesc& dw, const TmaDesc& dc
     case EPI_GELU: return launch_one<BN, EPI_GELU>(da, dw, dc, g, s);
     case EPI_RESIDUAL: return launch_one<BN, EPI_RESIDUAL>(da, dw, dc, g, s);
     case EPI_TABLE: return launch_one<BN, EPI_TABLE>(da, dw, dc, g, s);
+    case EPI_SWIGLU:
+      // gate / up pairs are 32-column chunks of full 256-wide tiles
+      if constexpr (BN == 256) { if (g.N % 256 == 0) return launch_one<BN, EPI_SWIGLU>(da, dw, dc, g, s); }
+      return cudaErrorInvalidValue;
   }
   return cudaErrorInvalidValue;
 }

@@ -14,8 +14,10 @@
 namespace et {
 namespace {
 
-// dst[n][K] (bf16) = src[k][n] (fp32)
-__global__ void transpose_weight_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int K, int N) {
+// dst[row(n)][K] (bf16) = src[k][n] (fp32).  row(n) = n, or, for a gated feed-forward weight with columns
+// [gate (gated_M) | up (gated_M)], the order the fused epilogue wants: tiles of 256 rows = 128 outputs, inside a
+// tile four groups of (32 gate rows, 32 up rows) of the same 32 outputs.
+__global__ void transpose_weight_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int K, int N, int gated_M) {
   __shared__ float tile[32][33];
   const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
   for (int i = threadIdx.y; i < 32; i += blockDim.y) {
@@ -25,7 +27,14 @@ __global__ void transpose_weight_kernel(const float* __restrict__ src, bf16* __r
   __syncthreads();
   for (int i = threadIdx.y; i < 32; i += blockDim.y) {
     const int n = n0 + i, k = k0 + threadIdx.x;
-    if (n < N && k < K) dst[(size_t)n * K + k] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+    if (n < N && k < K) {
+      int row = n;
+      if (gated_M > 0) {
+        const int up = n >= gated_M ? 1 : 0, j = n - up * gated_M;
+        row = (j >> 7) * 256 + ((j & 127) >> 5) * 64 + up * 32 + (j & 31);
+      }
+      dst[(size_t)row * K + k] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+    }
   }
 }
 
@@ -48,6 +57,7 @@ using namespace et;
 struct et_llm {
   et_llm_config cfg{};
   int device = 0, cap = 0;
+  bool fused_gate = false;
   int q_dim = 0, kv_dim = 0, qkv_dim = 0;
   std::string last_error;
   std::vector<void*> dev_allocs, host_allocs;
@@ -63,7 +73,7 @@ struct et_llm {
   float *X = nullptr, *logits = nullptr;
   bf16 *Xn = nullptr, *QKV = nullptr, *O = nullptr, *GU = nullptr, *Hm = nullptr, *Vb = nullptr, *P1 = nullptr, *Xl = nullptr;
   TmaDesc a_Xn, a_O, a_Hm, a_Vb, a_P1, a_Xl;        // operand maps
-  TmaDesc c_X, c_QKV, c_GU, c_P1, c_logits;          // output maps
+  TmaDesc c_X, c_QKV, c_GU, c_Hm, c_P1, c_logits;    // output maps
   int* ids = nullptr;                // device [cap]
   int* d_small = nullptr;            // [0] first token, [1] status
   int *h_ids = nullptr, *h_small = nullptr;          // pinned
@@ -179,6 +189,7 @@ et_status et_llm_create(const et_llm_config* config, const et_llm_weights* weigh
   m->q_dim = c.heads * c.head_dim; m->kv_dim = c.kv_heads * c.head_dim; m->qkv_dim = m->q_dim + 2 * m->kv_dim;
   const size_t qd = m->q_dim, qkv = m->qkv_dim;
   m->cap = (c.max_tokens + 255) / 256 * 256;          // whole row tiles: operand loads never leave the buffers
+  m->fused_gate = c.mlp_dim % 128 == 0;               // SwiGLU inside the gate/up layer's epilogue (whole 128-output tiles)
   const size_t cap = m->cap;
 
   // ---- weights: a staging buffer for host blobs, bf16 copies of the matrices, fp32 copies of the vectors
@@ -199,13 +210,13 @@ et_status et_llm_create(const et_llm_config* config, const et_llm_weights* weigh
     return ET_OK;
   };
   const char* err = nullptr;
-  auto matrix = [&](int K, int N, Dense* d) -> et_status {       // blob holds w [K][N]
+  auto matrix = [&](int K, int N, Dense* d, int gated_M = 0) -> et_status {       // blob holds w [K][N]
     const float* src = nullptr;
     et_status s2 = next((size_t)K * N, &src);
     if (s2 != ET_OK) return s2;
     if ((s2 = dalloc(m, &d->w, (size_t)N * K)) != ET_OK) return s2;
     ET_COUNT_LAUNCH();
-    transpose_weight_kernel<<<dim3(cdiv(N, 32), cdiv(K, 32)), dim3(32, 8)>>>(src, d->w, K, N);
+    transpose_weight_kernel<<<dim3(cdiv(N, 32), cdiv(K, 32)), dim3(32, 8)>>>(src, d->w, K, N, gated_M);
     if (cudaGetLastError() != cudaSuccess) return ET_ERR_CUDA;
     d->N = N; d->K = K;
     return make_tma_weight(&d->d, d->w, N, K, &err) ? ET_OK : ET_ERR_CUDA;
@@ -240,7 +251,7 @@ et_status et_llm_create(const et_llm_config* config, const et_llm_weights* weigh
     if ((st = vector_f32(qkv, &l.bqkv)) != ET_OK) return bail2(st);
     if ((st = matrix((int)qd, (int)H, &l.o)) != ET_OK) return bail2(st);
     if ((st = vector_f32(H, &l.rms2_g)) != ET_OK) return bail2(st);
-    if ((st = matrix((int)H, (int)(2 * M), &l.gu)) != ET_OK) return bail2(st);
+    if ((st = matrix((int)H, (int)(2 * M), &l.gu, m->fused_gate ? (int)M : 0)) != ET_OK) return bail2(st);
     if ((st = matrix((int)M, (int)H, &l.down)) != ET_OK) return bail2(st);
   }
   if ((st = vector_f32(H, &m->final_g)) != ET_OK) return bail2(st);
@@ -266,7 +277,7 @@ et_status et_llm_create(const et_llm_config* config, const et_llm_weights* weigh
     cudaMemset((ptr), 0, (count) * sizeof(*(ptr)));                      \
   } while (0)
   LLM_A(m->X, cap * H); LLM_A(m->Xn, cap * H); LLM_A(m->QKV, cap * qkv); LLM_A(m->O, cap * qd);
-  LLM_A(m->GU, cap * 2 * M); LLM_A(m->Hm, cap * M); LLM_A(m->Vb, cap * vh); LLM_A(m->P1, cap * H);
+  LLM_A(m->GU, m->fused_gate ? 8 : cap * 2 * M); LLM_A(m->Hm, cap * M); LLM_A(m->Vb, cap * vh); LLM_A(m->P1, cap * H);
   LLM_A(m->Xl, 256 * H); LLM_A(m->logits, 32 * V); LLM_A(m->ids, cap); LLM_A(m->d_small, (size_t)4);
 #undef LLM_A
   void* hp = nullptr;
@@ -279,7 +290,8 @@ et_status et_llm_create(const et_llm_config* config, const et_llm_weights* weigh
             make_tma_2d_bf16(&m->a_Hm, m->Hm, cap, M, 128, &err) && make_tma_2d_bf16(&m->a_Vb, m->Vb, cap, vh, 128, &err) &&
             make_tma_2d_bf16(&m->a_P1, m->P1, cap, H, 128, &err) && make_tma_2d_bf16(&m->a_Xl, m->Xl, 256, H, 128, &err) &&
             make_tma_out(&m->c_X, m->X, cap, H, true, &err) && make_tma_out(&m->c_QKV, m->QKV, cap, qkv, false, &err) &&
-            make_tma_out(&m->c_GU, m->GU, cap, 2 * M, false, &err) && make_tma_out(&m->c_P1, m->P1, cap, H, false, &err) &&
+            (m->fused_gate ? make_tma_out(&m->c_Hm, m->Hm, cap, M, false, &err) : make_tma_out(&m->c_GU, m->GU, cap, 2 * M, false, &err)) &&
+            make_tma_out(&m->c_P1, m->P1, cap, H, false, &err) &&
             make_tma_out(&m->c_logits, m->logits, 32, V, true, &err);
   if (!ok) return bail(lfail(m, ET_ERR_CUDA, err ? err : "tensor map"));
   if (cudaDeviceSynchronize() != cudaSuccess) return bail(ET_ERR_CUDA);
@@ -350,8 +362,12 @@ et_status et_llm_prefill(et_llm* m, const int* prefix_ids_host, int n_prefix, co
     SPAN(ET_LLM_ATTENTION, LLM_CUDA(m, launch_attention_causal(attn_map, m->O, 1, n, c.heads, c.kv_heads, m->d_small + 1, s)));
     SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_O, l.o, m->c_X, nullptr, m->X, n, EPI_RESIDUAL, s)));
     SPAN(ET_LLM_NORM, launch_rmsnorm(m->X, l.rms2_g, c.rms_eps, m->Xn, n, H, s));
-    SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_Xn, l.gu, m->c_GU, nullptr, m->GU, n, EPI_STORE, s)));
-    SPAN(ET_LLM_SWIGLU, launch_swiglu(m->GU, m->Hm, n, Mlp, s));
+    if (m->fused_gate) {
+      SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_Xn, l.gu, m->c_Hm, nullptr, m->Hm, n, EPI_SWIGLU, s)));
+    } else {
+      SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_Xn, l.gu, m->c_GU, nullptr, m->GU, n, EPI_STORE, s)));
+      SPAN(ET_LLM_SWIGLU, launch_swiglu(m->GU, m->Hm, n, Mlp, s));
+    }
     SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_Hm, l.down, m->c_X, nullptr, m->X, n, EPI_RESIDUAL, s)));
   }
 

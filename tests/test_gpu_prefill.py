@@ -79,6 +79,29 @@ def test_swiglu(B, rows, M):
     _close_bf16(h, P.silu(ref_in[:, :M]) * ref_in[:, M:], ulps=1.5)
 
 
+@pytest.mark.parametrize("rows,K,M", [(300, 256, 128), (1000, 512, 1408), (77, 64, 256)])
+def test_gated_dense_layer(B, rows, K, M):
+    """Dense layer with the SwiGLU epilogue: weight rows in the interleaved order, output silu(gate) * up."""
+    import torch
+    rng = np.random.default_rng(K + M)
+    a, a_ref = _bf16(rng.standard_normal((rows, K)))
+    wg, wg_ref = _bf16(rng.standard_normal((M, K)) / np.sqrt(K))        # [out][in]
+    wu, wu_ref = _bf16(rng.standard_normal((M, K)) / np.sqrt(K))
+    j = np.arange(M)
+    row_gate = (j >> 7) * 256 + ((j & 127) >> 5) * 64 + (j & 31)
+    w = torch.empty((2 * M, K), dtype=torch.bfloat16, device="cuda")
+    w[torch.from_numpy(row_gate).cuda()] = wg
+    w[torch.from_numpy(row_gate + 32).cuda()] = wu
+    bias = torch.zeros(2 * M, dtype=torch.float32, device="cuda")
+    h, status = B.et_linear_bf16(a, w, bias, epilogue=4)
+    assert int(status.item()) == 0 and tuple(h.shape) == (rows, M)
+    ref = P.silu(a_ref @ wg_ref.T) * (a_ref @ wu_ref.T)
+    got = h.float().cpu().numpy().astype(np.float64)
+    assert np.abs(got - ref).max() <= 1.5 * BF16_ULP * np.abs(ref).max() + 1e-5, f"error {np.abs(got - ref).max():.3e}"
+    err = np.abs(got - ref)
+    assert (err <= 2 * BF16_ULP * np.abs(ref) + 2e-3).all()
+
+
 @pytest.mark.parametrize("n_seq,L,heads,kv", [(1, 1, 1, 1), (1, 100, 2, 1), (1, 128, 1, 1), (1, 129, 2, 2), (1, 300, 4, 2),
                                               (2, 257, 2, 2), (1, 777, 4, 1), (3, 64, 7, 1), (1, 1500, 2, 1)])
 def test_attention_causal(B, n_seq, L, heads, kv):
