@@ -103,7 +103,8 @@ ET_API et_status et_rmsnorm(const float* x_dev, const float* g_dev, float eps, v
 /* Rotary position embedding, rotate-half form, in place on the Q and K parts of packed bf16 rows
  * [rows][(heads + 2*kv_heads)*head_dim]; row r has position r % L; element i < head_dim/2 of a head pairs
  * with i + head_dim/2 and the pair turns by position * theta^(-2i/head_dim).  head_dim % 16 == 0, <= 256.
- * Allocates and frees a table of head_dim/2 doubles (synchronises the stream). */
+ * Allocates and frees its table of angles (min(L, rows) * head_dim/2 cosine / sine pairs) and synchronises the
+ * stream; the model keeps such a table for its whole capacity instead. */
 ET_API et_status et_rope(void* qkv_dev, int rows, int L, int heads, int kv_heads, int head_dim, float theta, void* cuda_stream);
 
 /* h[r][j] = silu(gu[r][j]) * gu[r][M + j]; gu bf16 [rows][2M], h bf16 [rows][M]; M % 8 == 0. */

@@ -123,8 +123,10 @@ cudaError_t launch_attention_causal(const TmaDesc& map, bf16* out, int n_seq, in
 // y = x * rsqrt(mean(x^2) + eps) * g, rows [rows][D] fp32 -> bf16
 void launch_rmsnorm(const float* x, const float* g, float eps, bf16* y, int rows, int D, cudaStream_t s);
 // rotate-half rotary embedding in place on the Q and K parts of packed rows [rows][(heads + 2*kv_heads)*dh];
-// the position of a row is row % L; inv_turns [dh/2] (device, double) = theta^(-2i/dh) / (2 pi)
-void launch_rope(bf16* qkv, int rows, int L, int heads, int kv_heads, int dh, const double* inv_turns, cudaStream_t s);
+// the position of a row is row % L; table [>= L][dh/2] holds (cos, sin) of position * theta^(-2i/dh), filled by
+// launch_rope_table from inv_turns [dh/2] (device, double) = theta^(-2i/dh) / (2 pi)
+void launch_rope_table(float2* table, int L, int dh, const double* inv_turns, cudaStream_t s);
+void launch_rope(bf16* qkv, int rows, int L, int heads, int kv_heads, int dh, const float2* table, cudaStream_t s);
 // h[r][j] = silu(gu[r][j]) * gu[r][M + j]
 void launch_swiglu(const bf16* gu, bf16* h, int rows, int M, cudaStream_t s);
 // x[r][:] = table[ids[r]][:]  (bf16 table -> fp32 rows)

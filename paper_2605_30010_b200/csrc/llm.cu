@@ -69,6 +69,7 @@ struct et_llm {
   std::vector<LlmLayer> layers;
   float* zeros = nullptr;            // bias of the layers that have none
   double* inv_turns = nullptr;       // [head_dim/2] rotary frequencies in turns per position
+  float2* rope_table = nullptr;      // [cap][head_dim/2] (cos, sin) of every position
 
   float *X = nullptr, *logits = nullptr;
   bf16 *Xn = nullptr, *QKV = nullptr, *O = nullptr, *GU = nullptr, *Hm = nullptr, *Vb = nullptr, *P1 = nullptr, *Xl = nullptr;
@@ -268,6 +269,8 @@ et_status et_llm_create(const et_llm_config* config, const et_llm_weights* weigh
     for (int i = 0; i < half; ++i) t[i] = pow((double)c.rope_theta, -2.0 * i / (double)c.head_dim) / (2.0 * M_PI);
     if ((st = dalloc(m, &m->inv_turns, (size_t)half)) != ET_OK) return bail(st);
     if (cudaMemcpy(m->inv_turns, t.data(), half * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess) return bail(ET_ERR_CUDA);
+    if ((st = dalloc(m, &m->rope_table, cap * half)) != ET_OK) return bail(st);
+    launch_rope_table(m->rope_table, (int)cap, c.head_dim, m->inv_turns, 0);
   }
 
   // ---- activations (zeroed once: rows beyond the live count are read, never stored, by tile loads)
@@ -358,7 +361,7 @@ et_status et_llm_prefill(et_llm* m, const int* prefix_ids_host, int n_prefix, co
   for (const LlmLayer& l : m->layers) {
     SPAN(ET_LLM_NORM, launch_rmsnorm(m->X, l.rms1_g, c.rms_eps, m->Xn, n, H, s));
     SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_Xn, l.qkv, m->c_QKV, l.bqkv, m->QKV, n, EPI_STORE, s)));
-    SPAN(ET_LLM_ROPE, launch_rope(m->QKV, n, n, c.heads, c.kv_heads, c.head_dim, m->inv_turns, s));
+    SPAN(ET_LLM_ROPE, launch_rope(m->QKV, n, n, c.heads, c.kv_heads, c.head_dim, m->rope_table, s));
     SPAN(ET_LLM_ATTENTION, LLM_CUDA(m, launch_attention_causal(attn_map, m->O, 1, n, c.heads, c.kv_heads, m->d_small + 1, s)));
     SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_O, l.o, m->c_X, nullptr, m->X, n, EPI_RESIDUAL, s)));
     SPAN(ET_LLM_NORM, launch_rmsnorm(m->X, l.rms2_g, c.rms_eps, m->Xn, n, H, s));
@@ -427,12 +430,15 @@ et_status et_rope(void* qkv_dev, int rows, int L, int heads, int kv_heads, int h
   const int half = head_dim / 2;
   std::vector<double> t(half);
   for (int i = 0; i < half; ++i) t[i] = pow((double)theta, -2.0 * i / (double)head_dim) / (2.0 * M_PI);
+  const int Lt = L < rows ? L : rows;                     // positions that occur
   double* dev = nullptr;
-  if (cudaMalloc(&dev, half * sizeof(double)) != cudaSuccess) return ET_ERR_OOM;
+  if (cudaMalloc(&dev, half * sizeof(double) + (size_t)Lt * half * sizeof(float2)) != cudaSuccess) return ET_ERR_OOM;
+  float2* table = reinterpret_cast<float2*>(dev + half);
   cudaStream_t s = (cudaStream_t)cuda_stream;
   cudaError_t e = cudaMemcpyAsync(dev, t.data(), half * sizeof(double), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) {
-    launch_rope((bf16*)qkv_dev, rows, L, heads, kv_heads, head_dim, dev, s);
+    launch_rope_table(table, Lt, head_dim, dev, s);
+    launch_rope((bf16*)qkv_dev, rows, L, heads, kv_heads, head_dim, table, s);
     e = cudaGetLastError();
   }
   const cudaError_t e2 = cudaStreamSynchronize(s);

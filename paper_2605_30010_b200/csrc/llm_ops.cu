@@ -11,7 +11,7 @@ namespace {
 // RMSNorm: one warp per row, the row in registers (one read of x), fp32 statistics.
 // ---------------------------------------------------------------------------------------------
 template <int NV>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ g, float eps, bf16* __restrict__ y, int rows, int D) {
   const int warps_per_block = blockDim.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -38,13 +38,28 @@ rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ g, float e
 
 // ---------------------------------------------------------------------------------------------
 // Rotary embedding, rotate-half form: element i < dh/2 of a head pairs with element i + dh/2; the pair
-// is turned by pos * theta^(-2i/dh).  One thread handles 8 consecutive i of one (row, head): two
-// 16-byte loads and stores.  inv_turns[i] = theta^(-2i/dh) / (2 pi) comes from the host in double precision;
-// the angle is reduced to a fraction of a turn in double precision (positions reach 10^4 and more, where a
-// single-precision product loses that fraction), sine and cosine are fp32.
+// is turned by pos * theta^(-2i/dh).  The (cos, sin) of every (position, i) are tabulated once per model
+// (rope_table_kernel: the angle is reduced to a fraction of a turn in double precision, since positions reach
+// 10^4 and more, where a single-precision product loses that fraction; inv_turns[i] = theta^(-2i/dh) / (2 pi)
+// comes from the host in double precision).  The rotation itself then only streams: one thread handles 8
+// consecutive i of one (row, head), two 16-byte loads and stores plus 64 bytes of table from L2.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-rope_kernel(bf16* __restrict__ qkv, int rows, int L, int rot_heads, int row_elems, int dh, const double* __restrict__ inv_turns) {
+rope_table_kernel(float2* __restrict__ table, int L, int half, const double* __restrict__ inv_turns) {
+  const long long total = (long long)L * half;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total; idx += (long long)gridDim.x * blockDim.x) {
+    const int i = (int)(idx % half);
+    const long long pos = idx / half;
+    const double turns = (double)pos * inv_turns[i];                          // angle / 2 pi
+    const float frac = (float)(turns - floor(turns));
+    float sn, cs;
+    sincospif(2.f * frac, &sn, &cs);
+    table[idx] = make_float2(cs, sn);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+rope_kernel(bf16* __restrict__ qkv, int rows, int L, int rot_heads, int row_elems, int dh, const float2* __restrict__ table) {
   const int half = dh >> 1, chunks = half >> 3;
   const long long total = (long long)rows * rot_heads * chunks;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total; idx += (long long)gridDim.x * blockDim.x) {
@@ -54,23 +69,15 @@ rope_kernel(bf16* __restrict__ qkv, int rows, int L, int rot_heads, int row_elem
     const int pos = row % L;
     bf16* p = qkv + (size_t)row * row_elems + (size_t)h * dh + c * 8;
     uint4 a4 = *reinterpret_cast<const uint4*>(p), b4 = *reinterpret_cast<const uint4*>(p + half);
+    const float4* t4 = reinterpret_cast<const float4*>(table + (size_t)pos * half + c * 8);     // (cos, sin) x 2 per float4
     __nv_bfloat162* a2 = reinterpret_cast<__nv_bfloat162*>(&a4);
     __nv_bfloat162* b2 = reinterpret_cast<__nv_bfloat162*>(&b4);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      float2 a = __bfloat1622float2(a2[k]), b = __bfloat1622float2(b2[k]);
-      float sn[2], cs[2];
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int i = c * 8 + 2 * k + e;
-        const double turns = (double)pos * __ldg(inv_turns + i);               // angle / 2 pi
-        const float frac = (float)(turns - floor(turns));
-        sincospif(2.f * frac, &sn[e], &cs[e]);
-      }
-      const float2 ra = make_float2(a.x * cs[0] - b.x * sn[0], a.y * cs[1] - b.y * sn[1]);
-      const float2 rb = make_float2(b.x * cs[0] + a.x * sn[0], b.y * cs[1] + a.y * sn[1]);
-      a2[k] = __floats2bfloat162_rn(ra.x, ra.y);
-      b2[k] = __floats2bfloat162_rn(rb.x, rb.y);
+      const float2 a = __bfloat1622float2(a2[k]), b = __bfloat1622float2(b2[k]);
+      const float4 t = __ldg(t4 + k);                       // cos0, sin0, cos1, sin1
+      a2[k] = __floats2bfloat162_rn(a.x * t.x - b.x * t.y, a.y * t.z - b.y * t.w);
+      b2[k] = __floats2bfloat162_rn(b.x * t.x + a.x * t.y, b.y * t.z + a.y * t.w);
     }
     *reinterpret_cast<uint4*>(p) = a4;
     *reinterpret_cast<uint4*>(p + half) = b4;
@@ -178,8 +185,10 @@ int grid_for(long long work_items, int threads) {
 void launch_rmsnorm(const float* x, const float* g, float eps, bf16* y, int rows, int D, cudaStream_t s) {
   if (rows <= 0) return;
   ET_COUNT_LAUNCH();
-  const int threads = 256, wpb = threads / 32;
-  const int blocks = std::min(cdiv(rows, wpb), 148 * 8);
+  // 4 warps per block: a 3584-wide row takes 112 registers per thread, and three small blocks fit an SM where
+  // one of 8 warps would
+  const int threads = 128, wpb = threads / 32;
+  const int blocks = std::min(cdiv(rows, wpb), 148 * 12);
   const int need = cdiv(D / 4, 32);
 #define ET_RMS(NV) rmsnorm_kernel<NV><<<blocks, threads, 0, s>>>(x, g, eps, y, rows, D)
   if (need <= 2) ET_RMS(2);
@@ -191,12 +200,18 @@ void launch_rmsnorm(const float* x, const float* g, float eps, bf16* y, int rows
 #undef ET_RMS
 }
 
-void launch_rope(bf16* qkv, int rows, int L, int heads, int kv_heads, int dh, const double* inv_turns, cudaStream_t s) {
+void launch_rope_table(float2* table, int L, int dh, const double* inv_turns, cudaStream_t s) {
+  if (L <= 0) return;
+  ET_COUNT_LAUNCH();
+  rope_table_kernel<<<grid_for((long long)L * (dh / 2), 256), 256, 0, s>>>(table, L, dh / 2, inv_turns);
+}
+
+void launch_rope(bf16* qkv, int rows, int L, int heads, int kv_heads, int dh, const float2* table, cudaStream_t s) {
   if (rows <= 0) return;
   ET_COUNT_LAUNCH();
   const int rot = heads + kv_heads;
   const long long items = (long long)rows * rot * (dh / 16);
-  rope_kernel<<<grid_for(items, 256), 256, 0, s>>>(qkv, rows, L, rot, (heads + 2 * kv_heads) * dh, dh, inv_turns);
+  rope_kernel<<<grid_for(items, 256), 256, 0, s>>>(qkv, rows, L, rot, (heads + 2 * kv_heads) * dh, dh, table);
 }
 
 void launch_swiglu(const bf16* gu, bf16* h, int rows, int M, cudaStream_t s) {
