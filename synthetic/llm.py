@@ -61,6 +61,10 @@ QWEN2_7B_1L = LlmShape(vision_hidden=1152, hidden=3584, num_layers=1, heads=28, 
                        mlp_dim=18944, vocab=1024)
 LLM_TINY = LlmShape(vision_hidden=64, hidden=256, num_layers=2, heads=2, kv_heads=1, head_dim=128, mlp_dim=512,
                     vocab=512, rope_theta=1e4)
+# mlp_dim not a multiple of 128 (the feed-forward gating runs as a kernel of its own) and as many key / value heads as
+# query heads (plain multi-head attention)
+LLM_ODD = LlmShape(vision_hidden=72, hidden=384, num_layers=2, heads=3, kv_heads=3, head_dim=128, mlp_dim=328, vocab=264,
+                   rope_theta=5e5, gelu_tanh=0)
 LLM_SMALL = LlmShape(vision_hidden=1152, hidden=512, num_layers=3, heads=4, kv_heads=2, head_dim=128, mlp_dim=1408,
                      vocab=1000)
 

@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 
 from oracle import prefill_oracle as P
-from synthetic.llm import (LLM_SMALL, LLM_TINY, QWEN2_7B, QWEN2_7B_1L, LlmShape, make_llm_weights, make_llm_weights_device,
+from synthetic.llm import (LLM_ODD, LLM_SMALL, LLM_TINY, QWEN2_7B, QWEN2_7B_1L, LlmShape, make_llm_weights, make_llm_weights_device,
                            make_prompt, make_visual_tokens)
 from tests import helpers as H
 
@@ -154,7 +154,8 @@ def _check_prefill(r, r2, ref):
 
 
 @pytest.mark.parametrize("shape,n_prefix,n_vis,n_suffix", [(LLM_TINY, 5, 300, 9), (LLM_TINY, 0, 130, 0), (LLM_TINY, 3, 0, 4),
-                                                           (LLM_SMALL, 14, 500, 21), (LLM_SMALL, 1, 255, 0)])
+                                                           (LLM_SMALL, 14, 500, 21), (LLM_SMALL, 1, 255, 0),
+                                                           (LLM_ODD, 7, 290, 3), (LLM_ODD, 1, 0, 0), (LLM_TINY, 0, 256, 0)])
 def test_prefill_small_models(B, shape, n_prefix, n_vis, n_suffix):
     blob = make_llm_weights(shape, 3)
     r, r2, ref = _run_prefill(B, shape, blob, n_prefix, n_vis, n_suffix, 1, np.float64)

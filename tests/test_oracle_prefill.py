@@ -8,7 +8,7 @@ import torch
 import torch.nn.functional as F
 
 from oracle import prefill_oracle as P
-from synthetic.llm import LLM_TINY, LlmShape, llm_blob_size, llm_weight_layout, make_llm_weights, make_prompt, make_visual_tokens
+from synthetic.llm import LLM_ODD, LLM_TINY, LlmShape, llm_blob_size, llm_weight_layout, make_llm_weights, make_prompt, make_visual_tokens
 
 SHAPE = LlmShape(vision_hidden=24, hidden=32, num_layers=2, heads=4, kv_heads=2, head_dim=8, mlp_dim=48, vocab=50,
                  rope_theta=100.0)
@@ -83,7 +83,8 @@ def _torch_prefill(shape, w, pre, vis, suf):
     if len(pre):
         parts.append(F.embedding(torch.from_numpy(pre.astype(np.int64)), t["embed"]))
     if len(vis):
-        h = F.gelu(F.linear(torch.from_numpy(vis.astype(np.float64)), t["proj_w1"].T, t["proj_b1"]), approximate="tanh")
+        h = F.gelu(F.linear(torch.from_numpy(vis.astype(np.float64)), t["proj_w1"].T, t["proj_b1"]),
+                   approximate="tanh" if shape.gelu_tanh else "none")
         parts.append(F.linear(h, t["proj_w2"].T, t["proj_b2"]))
     if len(suf):
         parts.append(F.embedding(torch.from_numpy(suf.astype(np.int64)), t["embed"]))
@@ -106,7 +107,7 @@ def _torch_prefill(shape, w, pre, vis, suf):
     return X.numpy(), F.linear(last, t["lm_head"].T)[0].numpy()
 
 
-@pytest.mark.parametrize("shape", [SHAPE, LLM_TINY])
+@pytest.mark.parametrize("shape", [SHAPE, LLM_TINY, LLM_ODD])
 def test_prefill_against_torch_composition(shape):
     blob, w, pre, vis, suf = _setup(shape)
     got = P.prefill(shape, w, pre, vis, suf, want_hidden=True)
