@@ -29,6 +29,8 @@ constexpr int ATOM_BYTES = 128 * 128;   // 128 rows x 64 bf16, 128-byte swizzle
 constexpr int TILE_BYTES = 2 * ATOM_BYTES;   // 128 rows x 128 bf16: columns 0..63, then 64..127
 constexpr int ATT_THREADS = 384;        // warps 0..7 softmax, 8 TMA, 9 MMA, 10..11 idle (complete the third warpgroup)
 constexpr int SOFTMAX_REGS = 200, CONTROL_REGS = 80;
+// (nothing checks that a role's code fits its budget -- a path that needs more computes garbage silently; the
+// parity tests validate these numbers)
 // setmaxnreg.inc blocks until the registers exist: the budgets must fit into what the CTA was launched with
 constexpr int LAUNCH_REGS = 160;
 static_assert(SOFTMAX_REGS * 256 + CONTROL_REGS * 128 <= LAUNCH_REGS * ATT_THREADS, "register budgets exceed the CTA's allocation");

@@ -37,6 +37,9 @@ constexpr int MAIN_BYTES = 128 * 128;   // 128 rows x 64 bf16, 128-byte swizzle
 constexpr int TAIL_BYTES = 128 * 16;    // 128 rows x 8 bf16, rows 16 bytes apart
 constexpr int ATT_THREADS = 384;         // warps 0..7 softmax, 8 TMA, 9 MMA, 10..11 idle (complete the third warpgroup)
 constexpr int SOFTMAX_REGS = 200, CONTROL_REGS = 80;   // per-thread register budgets after setmaxnreg
+// Nothing checks that a role's code fits its budget: a path that needs more registers than it kept runs on with
+// lost values and computes garbage without any error (seen when the MMA path was given a run-time group index).
+// The parity tests are what validates these two numbers.
 // setmaxnreg.inc blocks until the registers exist: the budgets must fit into what the CTA was launched with,
 // which is at least LAUNCH_REGS per thread (the kernel is compiled for exactly one CTA of ATT_THREADS per SM).
 constexpr int LAUNCH_REGS = 160;
