@@ -196,7 +196,7 @@ def run_downstream(args, wl, enc, dev_vids, offs, stream, peaks, torch, B):
     T, L = wl.total_frames, wl.shape.tokens_per_frame
     n_text = (14, 40)
     blob = make_llm_weights_device(shape, 77)
-    llm = B.LanguageModel(shape, blob, max_tokens=T * L + sum(n_text))
+    llm = B.LanguageModel(shape, blob, max_tokens=T * L + sum(n_text), keep_kv_cache=True)      # a prefill that decoding could follow
     del blob
     torch.cuda.empty_cache()
     pre, suf = make_prompt(shape, n_text[0], n_text[1], 77)

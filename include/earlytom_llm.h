@@ -40,6 +40,7 @@ typedef struct {
   float rope_theta;
   int gelu_tanh;          /* projector activation: 1 tanh approximation, 0 erf form */
   int max_tokens;         /* workspace capacity: sequence length of one call */
+  int keep_kv_cache;      /* 1: every layer's keys (after the rotary embedding) and values are kept for decoding */
 } et_llm_config;
 
 /* fp32 blob in this fixed order (row-major, a linear layer is y = x W + b with W [in][out]):
@@ -65,6 +66,10 @@ typedef struct {
   int first_token;           /* argmax of the logits of the last position (lowest id among equals) */
   const float* logits;       /* device fp32 [vocab], last position */
   const float* hidden;       /* device fp32 [n_tokens][hidden]: residual stream after the last layer */
+  const void* kv_cache;      /* NULL unless keep_kv_cache: device bf16 [num_layers][kv_cache_rows][2*kv_heads*head_dim],
+                                row p of a layer = [keys of position p, rotated | values of position p]; rows >= n_tokens
+                                are stale */
+  int kv_cache_rows;         /* row count of one layer's slab (the capacity, a multiple of 256) */
 } et_llm_result;
 
 /* Errors: ET_ERR_SHAPE for widths the kernels do not cover, ET_ERR_WEIGHTS when count does not match the

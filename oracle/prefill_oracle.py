@@ -112,8 +112,9 @@ def projector(tokens: np.ndarray, w, shape) -> np.ndarray:
     return h @ w["proj_w2"].astype(dt) + w["proj_b2"].astype(dt)
 
 
-def decoder_layer(X: np.ndarray, w, layer: int, shape) -> np.ndarray:
-    """One pre-norm decoder block on the whole sequence X [n, hidden]."""
+def decoder_layer(X: np.ndarray, w, layer: int, shape, kv_out: Optional[list] = None) -> np.ndarray:
+    """One pre-norm decoder block on the whole sequence X [n, hidden].  kv_out, if given, receives this layer's
+    (rotated keys [n, kv_heads, d], values [n, kv_heads, d]): what a decoder would cache."""
     p = f"l{layer}."
     n, dt = X.shape[0], X.dtype
     H, KV, d = shape.heads, shape.kv_heads, shape.head_dim
@@ -123,7 +124,10 @@ def decoder_layer(X: np.ndarray, w, layer: int, shape) -> np.ndarray:
     k = qkv[:, H * d:(H + KV) * d].reshape(n, KV, d)
     v = qkv[:, (H + KV) * d:].reshape(n, KV, d)
     pos = np.arange(n)
-    ctx = causal_gqa_attention(rope(q, pos, shape.rope_theta), rope(k, pos, shape.rope_theta), v)
+    k_rot = rope(k, pos, shape.rope_theta)
+    if kv_out is not None:
+        kv_out.append((k_rot.copy(), v.copy()))
+    ctx = causal_gqa_attention(rope(q, pos, shape.rope_theta), k_rot, v)
     X = X + ctx.reshape(n, H * d) @ w[p + "wo"].astype(dt)
     xn = rms_norm(X, w[p + "rms2_g"], shape.rms_eps)
     gu = xn @ w[p + "wgu"].astype(dt)
@@ -144,16 +148,17 @@ def assemble_sequence(shape, w, prefix_ids, visual_tokens: np.ndarray, suffix_id
 
 
 def prefill(shape, w, prefix_ids, visual_tokens: np.ndarray, suffix_ids, dtype=np.float64,
-            want_hidden: bool = False) -> dict:
+            want_hidden: bool = False, want_kv: bool = False) -> dict:
     """Prefill of the whole sequence; the logits of the last position give the first generated token."""
     X = assemble_sequence(shape, w, prefix_ids, visual_tokens, suffix_ids, dtype)
     embeds = X.copy() if want_hidden else None
+    kv = [] if want_kv else None
     for layer in range(shape.num_layers):
-        X = decoder_layer(X, w, layer, shape)
+        X = decoder_layer(X, w, layer, shape, kv)
     last = rms_norm(X[-1:], w["final_g"], shape.rms_eps)
     logits = (last @ w["lm_head"].astype(dtype))[0]
     return dict(logits=logits, first_token=int(np.argmax(logits)), last_hidden=X[-1].copy(),
-                hidden=X if want_hidden else None, embeds=embeds, n_tokens=X.shape[0])
+                hidden=X if want_hidden else None, embeds=embeds, n_tokens=X.shape[0], kv=kv)
 
 
 def prefill_flops(shape, n_tokens: int, n_vis: int) -> float:

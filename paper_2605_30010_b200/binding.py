@@ -97,7 +97,8 @@ class et_profile(C.Structure):
 class et_llm_config(C.Structure):
     _fields_ = [("vision_hidden", C.c_int), ("hidden", C.c_int), ("num_layers", C.c_int), ("heads", C.c_int),
                 ("kv_heads", C.c_int), ("head_dim", C.c_int), ("mlp_dim", C.c_int), ("vocab", C.c_int),
-                ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("gelu_tanh", C.c_int), ("max_tokens", C.c_int)]
+                ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("gelu_tanh", C.c_int), ("max_tokens", C.c_int),
+                ("keep_kv_cache", C.c_int)]
 
 
 class et_llm_weights(C.Structure):
@@ -105,7 +106,8 @@ class et_llm_weights(C.Structure):
 
 
 class et_llm_result(C.Structure):
-    _fields_ = [("n_tokens", C.c_int), ("first_token", C.c_int), ("logits", C.c_void_p), ("hidden", C.c_void_p)]
+    _fields_ = [("n_tokens", C.c_int), ("first_token", C.c_int), ("logits", C.c_void_p), ("hidden", C.c_void_p),
+                ("kv_cache", C.c_void_p), ("kv_cache_rows", C.c_int)]
 
 
 ET_LLM_CATS = 8
@@ -566,6 +568,7 @@ class PrefillResult:
     first_token: int
     logits: object        # torch fp32 [vocab] (copy)
     hidden: object        # torch fp32 [n_tokens, hidden] (copy) or None
+    kv_cache: object = None   # torch bf16 [layers, n_tokens, 2*kv_heads*head_dim] (copy), on request
 
 
 def et_llm_create(cfg: et_llm_config, weights) -> C.c_void_p:
@@ -588,10 +591,10 @@ def et_llm_destroy(handle) -> None:
 class LanguageModel:
     """Owns an et_llm*.  `shape` is any object with the architecture fields of et_llm_config."""
 
-    def __init__(self, shape, weights, max_tokens: int):
+    def __init__(self, shape, weights, max_tokens: int, keep_kv_cache: bool = False):
         cfg = et_llm_config(shape.vision_hidden, shape.hidden, shape.num_layers, shape.heads, shape.kv_heads, shape.head_dim,
                             shape.mlp_dim, shape.vocab, float(shape.rms_eps), float(shape.rope_theta), int(shape.gelu_tanh),
-                            int(max_tokens))
+                            int(max_tokens), 1 if keep_kv_cache else 0)
         self.handle = et_llm_create(cfg, weights)
         self.shape = shape
 
@@ -606,8 +609,8 @@ class LanguageModel:
         except Exception:
             pass
 
-    def prefill(self, prefix_ids, visual_tokens, suffix_ids, want_hidden=False, stream=None) -> PrefillResult:
-        return et_llm_prefill(self, prefix_ids, visual_tokens, suffix_ids, want_hidden, stream)
+    def prefill(self, prefix_ids, visual_tokens, suffix_ids, want_hidden=False, stream=None, want_kv=False) -> PrefillResult:
+        return et_llm_prefill(self, prefix_ids, visual_tokens, suffix_ids, want_hidden, stream, want_kv=want_kv)
 
 
 def _ids(a):
@@ -616,7 +619,7 @@ def _ids(a):
 
 
 def et_llm_prefill(llm: LanguageModel, prefix_ids, visual_tokens, suffix_ids, want_hidden=False, stream=None,
-                   copy_logits=True) -> PrefillResult:
+                   copy_logits=True, want_kv=False) -> PrefillResult:
     """visual_tokens: torch fp32 CUDA [n_visual, vision_hidden] (or None)."""
     pre, pre_p = _ids(prefix_ids)
     suf, suf_p = _ids(suffix_ids)
@@ -632,7 +635,16 @@ def et_llm_prefill(llm: LanguageModel, prefix_ids, visual_tokens, suffix_ids, wa
         raise EarlyTomError(st, lib().et_llm_last_error(llm.handle).decode())
     logits = _dev_tensor(r.logits, (llm.shape.vocab,), "<f4") if copy_logits else None
     hidden = _dev_tensor(r.hidden, (r.n_tokens, llm.shape.hidden), "<f4") if want_hidden else None
-    return PrefillResult(r.n_tokens, r.first_token, logits, hidden)
+    kv = None
+    if want_kv:
+        if not r.kv_cache:
+            raise EarlyTomError(1, "the model was created without keep_kv_cache")
+        import torch
+        sh = llm.shape
+        full = torch.as_tensor(_DevView(r.kv_cache, (sh.num_layers, r.kv_cache_rows, 2 * sh.kv_heads * sh.head_dim * 2), "|u1"),
+                               device="cuda")
+        kv = full[:, :r.n_tokens].clone().view(torch.bfloat16)
+    return PrefillResult(r.n_tokens, r.first_token, logits, hidden, kv)
 
 
 def et_llm_profile_enable(llm: LanguageModel, on: bool) -> None:

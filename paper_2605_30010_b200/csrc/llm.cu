@@ -70,6 +70,7 @@ struct et_llm {
   float* zeros = nullptr;            // bias of the layers that have none
   double* inv_turns = nullptr;       // [head_dim/2] rotary frequencies in turns per position
   float2* rope_table = nullptr;      // [cap][head_dim/2] (cos, sin) of every position
+  bf16* kv_cache = nullptr;          // [layers][cap][2*kv_dim] when the model keeps keys and values
 
   float *X = nullptr, *logits = nullptr;
   bf16 *Xn = nullptr, *QKV = nullptr, *O = nullptr, *GU = nullptr, *Hm = nullptr, *Vb = nullptr, *P1 = nullptr, *Xl = nullptr;
@@ -150,6 +151,7 @@ et_status validate(const et_llm_config* c) {
   if (c->mlp_dim < 8 || c->mlp_dim % 8 || c->vocab < 8 || c->vocab % 8) return ET_ERR_SHAPE;
   if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return ET_ERR_INVALID_ARG;
   if (c->max_tokens < 1 || c->max_tokens > (1 << 20)) return ET_ERR_INVALID_ARG;
+  if (c->keep_kv_cache != 0 && c->keep_kv_cache != 1) return ET_ERR_INVALID_ARG;
   return ET_OK;
 }
 
@@ -281,6 +283,7 @@ et_status et_llm_create(const et_llm_config* config, const et_llm_weights* weigh
   } while (0)
   LLM_A(m->X, cap * H); LLM_A(m->Xn, cap * H); LLM_A(m->QKV, cap * qkv); LLM_A(m->O, cap * qd);
   LLM_A(m->GU, m->fused_gate ? 8 : cap * 2 * M); LLM_A(m->Hm, cap * M); LLM_A(m->Vb, cap * vh); LLM_A(m->P1, cap * H);
+  if (c.keep_kv_cache) LLM_A(m->kv_cache, (size_t)c.num_layers * cap * 2 * m->kv_dim);
   LLM_A(m->Xl, 256 * H); LLM_A(m->logits, 32 * V); LLM_A(m->ids, cap); LLM_A(m->d_small, (size_t)4);
 #undef LLM_A
   void* hp = nullptr;
@@ -358,10 +361,17 @@ et_status et_llm_prefill(et_llm* m, const int* prefix_ids_host, int n_prefix, co
   // ---- decoder layers
   TmaDesc attn_map;
   if (!make_causal_attention_map(&attn_map, m->QKV, n, c.heads, c.kv_heads)) return lfail(m, ET_ERR_CUDA, "tensor map of the attention operands");
+  int layer_index = 0;
   for (const LlmLayer& l : m->layers) {
     SPAN(ET_LLM_NORM, launch_rmsnorm(m->X, l.rms1_g, c.rms_eps, m->Xn, n, H, s));
     SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_Xn, l.qkv, m->c_QKV, l.bqkv, m->QKV, n, EPI_STORE, s)));
     SPAN(ET_LLM_ROPE, launch_rope(m->QKV, n, n, c.heads, c.kv_heads, c.head_dim, m->rope_table, s));
+    if (m->kv_cache) {      // the K | V columns of the packed rows, as they are after the rotation
+      const size_t kvw = (size_t)2 * m->kv_dim * sizeof(bf16);
+      SPAN(ET_LLM_ROPE, LLM_CUDA(m, cudaMemcpy2DAsync(m->kv_cache + (size_t)layer_index * m->cap * 2 * m->kv_dim, kvw, m->QKV + m->q_dim,
+                                                     (size_t)m->qkv_dim * sizeof(bf16), kvw, n, cudaMemcpyDeviceToDevice, s)));
+    }
+    ++layer_index;
     SPAN(ET_LLM_ATTENTION, LLM_CUDA(m, launch_attention_causal(attn_map, m->O, 1, n, c.heads, c.kv_heads, m->d_small + 1, s)));
     SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_O, l.o, m->c_X, nullptr, m->X, n, EPI_RESIDUAL, s)));
     SPAN(ET_LLM_NORM, launch_rmsnorm(m->X, l.rms2_g, c.rms_eps, m->Xn, n, H, s));
@@ -397,6 +407,7 @@ et_status et_llm_prefill(et_llm* m, const int* prefix_ids_host, int n_prefix, co
   }
   et_llm_result r{};
   r.n_tokens = n; r.first_token = m->h_small[0]; r.logits = m->logits; r.hidden = m->X;
+  r.kv_cache = m->kv_cache; r.kv_cache_rows = m->kv_cache ? m->cap : 0;
   *out = r;
   return ET_OK;
 }

@@ -34,7 +34,7 @@ def main():
 
     shape = replace(QWEN2_7B, num_layers=args.layers, vocab=args.vocab)
     blob = make_llm_weights_device(shape, 5)
-    llm = B.LanguageModel(shape, blob, max_tokens=args.visual_tokens + 64)
+    llm = B.LanguageModel(shape, blob, max_tokens=args.visual_tokens + 64, keep_kv_cache=True)
     del blob
     torch.cuda.empty_cache()
     pre, suf = make_prompt(shape, 14, 40, 6)

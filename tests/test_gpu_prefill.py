@@ -173,6 +173,33 @@ def test_prefill_one_layer_at_full_width(B):
     print(f"full width, one layer: n = {r.n_tokens}, hidden error {err:.2e}, logit error {lerr:.2e}")
 
 
+def test_kv_cache(B):
+    """Keys (after the rotary embedding) and values of every layer, as kept for decoding, against the oracle's."""
+    import torch
+    shape = LLM_SMALL
+    blob = make_llm_weights(shape, 3)
+    pre, suf = make_prompt(shape, 6, 11, 4)
+    vis = make_visual_tokens(shape, 300, 4)
+    llm = B.LanguageModel(shape, blob, max_tokens=400, keep_kv_cache=True)
+    plain = B.LanguageModel(shape, blob, max_tokens=400)
+    try:
+        r = llm.prefill(pre, torch.from_numpy(vis).cuda(), suf, want_hidden=True, want_kv=True)
+        r0 = plain.prefill(pre, torch.from_numpy(vis).cuda(), suf, want_hidden=True)
+        with pytest.raises(B.EarlyTomError):
+            plain.prefill(pre, torch.from_numpy(vis).cuda(), suf, want_kv=True)
+    finally:
+        llm.close(); plain.close()
+    assert torch.equal(r.hidden, r0.hidden), "keeping the cache must not change the result"
+    ref = P.prefill(shape, P.split_llm_weights(shape, blob), pre, vis, suf, want_kv=True)
+    n, kvd = r.n_tokens, shape.kv_heads * shape.head_dim
+    assert tuple(r.kv_cache.shape) == (shape.num_layers, n, 2 * kvd)
+    got = r.kv_cache.float().cpu().numpy()
+    for layer, (k, v) in enumerate(ref["kv"]):
+        ek = H.token_error(got[layer, :, :kvd], k.reshape(n, kvd))
+        ev = H.token_error(got[layer, :, kvd:], v.reshape(n, kvd))
+        assert ek <= BF16_TOL and ev <= BF16_TOL, f"layer {layer}: key error {ek:.3e}, value error {ev:.3e}"
+
+
 def test_errors(B):
     import torch
     shape = LLM_TINY

@@ -90,6 +90,7 @@ def _torch_prefill(shape, w, pre, vis, suf):
         parts.append(F.embedding(torch.from_numpy(suf.astype(np.int64)), t["embed"]))
     X = torch.cat(parts, dim=0)
     n, H, KV, d, M = X.shape[0], shape.heads, shape.kv_heads, shape.head_dim, shape.mlp_dim
+    kv = []
     for i in range(shape.num_layers):
         p = f"l{i}."
         xn = F.rms_norm(X, (shape.hidden,), t[p + "rms1_g"], eps=shape.rms_eps)
@@ -97,6 +98,7 @@ def _torch_prefill(shape, w, pre, vis, suf):
         q = _rope_complex(qkv[:, :H * d].reshape(n, H, d), shape.rope_theta)
         k = _rope_complex(qkv[:, H * d:(H + KV) * d].reshape(n, KV, d), shape.rope_theta)
         v = qkv[:, (H + KV) * d:].reshape(n, KV, d)
+        kv.append((k.numpy().copy(), v.numpy().copy()))
         ctx = F.scaled_dot_product_attention(q.transpose(0, 1)[None], k.transpose(0, 1)[None], v.transpose(0, 1)[None],
                                              is_causal=True, enable_gqa=True)[0].transpose(0, 1).reshape(n, H * d)
         X = X + F.linear(ctx, t[p + "wo"].T)
@@ -104,15 +106,19 @@ def _torch_prefill(shape, w, pre, vis, suf):
         gu = F.linear(xn, t[p + "wgu"].T)
         X = X + F.linear(F.silu(gu[:, :M]) * gu[:, M:], t[p + "wd"].T)
     last = F.rms_norm(X[-1:], (shape.hidden,), t["final_g"], eps=shape.rms_eps)
-    return X.numpy(), F.linear(last, t["lm_head"].T)[0].numpy()
+    return X.numpy(), F.linear(last, t["lm_head"].T)[0].numpy(), kv
 
 
 @pytest.mark.parametrize("shape", [SHAPE, LLM_TINY, LLM_ODD])
 def test_prefill_against_torch_composition(shape):
     blob, w, pre, vis, suf = _setup(shape)
-    got = P.prefill(shape, w, pre, vis, suf, want_hidden=True)
-    X, logits = _torch_prefill(shape, w, pre, vis, suf)
+    got = P.prefill(shape, w, pre, vis, suf, want_hidden=True, want_kv=True)
+    X, logits, kv = _torch_prefill(shape, w, pre, vis, suf)
     np.testing.assert_allclose(got["hidden"], X, rtol=1e-9, atol=1e-9)
+    assert len(got["kv"]) == shape.num_layers
+    for (k_o, v_o), (k_t, v_t) in zip(got["kv"], kv):         # what a decoder would cache: rotated keys, values
+        np.testing.assert_allclose(k_o, k_t, rtol=1e-9, atol=1e-9)
+        np.testing.assert_allclose(v_o, v_t, rtol=1e-9, atol=1e-9)
     np.testing.assert_allclose(got["logits"], logits, rtol=1e-9, atol=1e-9)
     assert got["first_token"] == int(np.argmax(logits)) and got["n_tokens"] == len(pre) + len(vis) + len(suf)
 
