@@ -132,6 +132,8 @@ void launch_swiglu(const bf16* gu, bf16* h, int rows, int M, cudaStream_t s);
 // x[r][:] = table[ids[r]][:]  (bf16 table -> fp32 rows)
 void launch_embed_rows(const bf16* table, const int* ids, float* x, int rows, int D, int vocab, cudaStream_t s);
 void launch_cast_bf16(const float* x, bf16* y, size_t count, cudaStream_t s);
+// dst[r][0..width) = src[r][0..width); width and both pitches in elements, multiples of 8; 16-byte aligned pointers
+void launch_copy_columns(const bf16* src, bf16* dst, int rows, int width, int src_pitch, int dst_pitch, cudaStream_t s);
 // first index of the maximum of x[0..n)
 void launch_argmax(const float* x, int n, int* out, cudaStream_t s);
 

@@ -366,11 +366,9 @@ et_status et_llm_prefill(et_llm* m, const int* prefix_ids_host, int n_prefix, co
     SPAN(ET_LLM_NORM, launch_rmsnorm(m->X, l.rms1_g, c.rms_eps, m->Xn, n, H, s));
     SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_Xn, l.qkv, m->c_QKV, l.bqkv, m->QKV, n, EPI_STORE, s)));
     SPAN(ET_LLM_ROPE, launch_rope(m->QKV, n, n, c.heads, c.kv_heads, c.head_dim, m->rope_table, s));
-    if (m->kv_cache) {      // the K | V columns of the packed rows, as they are after the rotation
-      const size_t kvw = (size_t)2 * m->kv_dim * sizeof(bf16);
-      SPAN(ET_LLM_ROPE, LLM_CUDA(m, cudaMemcpy2DAsync(m->kv_cache + (size_t)layer_index * m->cap * 2 * m->kv_dim, kvw, m->QKV + m->q_dim,
-                                                     (size_t)m->qkv_dim * sizeof(bf16), kvw, n, cudaMemcpyDeviceToDevice, s)));
-    }
+    if (m->kv_cache)        // the K | V columns of the packed rows, as they are after the rotation
+      SPAN(ET_LLM_ROPE, launch_copy_columns(m->QKV + m->q_dim, m->kv_cache + (size_t)layer_index * m->cap * 2 * m->kv_dim, n, 2 * m->kv_dim,
+                                           m->qkv_dim, 2 * m->kv_dim, s));
     ++layer_index;
     SPAN(ET_LLM_ATTENTION, LLM_CUDA(m, launch_attention_causal(attn_map, m->O, 1, n, c.heads, c.kv_heads, m->d_small + 1, s)));
     SPAN(ET_LLM_GEMM, LLM_TRY(dense(m, m->a_O, l.o, m->c_X, nullptr, m->X, n, EPI_RESIDUAL, s)));

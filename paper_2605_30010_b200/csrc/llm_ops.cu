@@ -126,6 +126,17 @@ embed_rows_kernel(const bf16* __restrict__ table, const int* __restrict__ ids, f
   }
 }
 
+// dst[r][0..w) = src[r][0..w) for row pitches given in 16-byte units (a column block of a wider matrix)
+__global__ void __launch_bounds__(256)
+copy_columns_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int rows, int w16, int src_pitch16, int dst_pitch16) {
+  const long long total = (long long)rows * w16;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total; idx += (long long)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % w16);
+    const long long r = idx / w16;
+    dst[r * dst_pitch16 + c] = __ldg(src + r * src_pitch16 + c);
+  }
+}
+
 __global__ void __launch_bounds__(256)
 cast_bf16_kernel(const float* __restrict__ x, bf16* __restrict__ y, size_t count) {
   const size_t n4 = count >> 2;
@@ -230,6 +241,13 @@ void launch_cast_bf16(const float* x, bf16* y, size_t count, cudaStream_t s) {
   if (count == 0) return;
   ET_COUNT_LAUNCH();
   cast_bf16_kernel<<<grid_for((long long)(count / 4 + 1), 256), 256, 0, s>>>(x, y, count);
+}
+
+void launch_copy_columns(const bf16* src, bf16* dst, int rows, int width, int src_pitch, int dst_pitch, cudaStream_t s) {
+  if (rows <= 0 || width <= 0) return;
+  ET_COUNT_LAUNCH();
+  copy_columns_kernel<<<grid_for((long long)rows * (width / 8), 256), 256, 0, s>>>(
+      reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), rows, width / 8, src_pitch / 8, dst_pitch / 8);
 }
 
 void launch_argmax(const float* x, int n, int* out, cudaStream_t s) {
