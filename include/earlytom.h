@@ -65,7 +65,7 @@ typedef struct {
   int gelu_tanh;        /* 1 = tanh approximation of GELU, 0 = erf form */
   int post_layernorm;   /* 1 = final LayerNorm applied to the kept tokens */
   int dtype;            /* et_dtype */
-  int max_frames_total; /* capacity: sum of frames over the videos of one call */
+  int max_frames_total; /* capacity: sum of frames over the videos of one call, at most 65535 */
   int max_videos;       /* capacity: videos per call */
 } et_config;
 
@@ -106,6 +106,10 @@ typedef struct {
   const et_forced_plan* forced_plan; /* NULL = decide */
   int want_trace;       /* 1 = fill et_result.trace */
   unsigned long long sample_seed; /* selection 3 only */
+  int window_mode;      /* local windows of a static frame (Eq. 6).  0: as printed, runs of w = floor(L/k) positions,
+                           M = ceil(L/w) windows (M >= k; M = L once k > L/2, i.e. static frames keep everything);
+                           1: k windows [floor(m*L/k), floor((m+1)*L/k)), so static and dynamic frames keep the same
+                           amount and the total is N*k ~ retain*B*L.  Both coincide when k divides L. */
 } et_params;
 
 /* Decision trace, host memory owned by the encoder.  Per merge layer i the arrays cover the list
@@ -257,9 +261,11 @@ ET_API et_status et_merge_frames(const float* x_dev, float* y_dev, int n_cap, in
 
 /* Paper Eq. 4 / Eq. 6: keep mask of N frames from scores [N][L]; frame f keeps its k_dev[f]
  * highest scores (ties to the lower index) when dynamic_dev[f] != 0, else the first maximum of
- * each window of width w_dev[f].  keep_dev bytes [N][L], count_dev int [N]. */
+ * each local window: runs of w_dev[f] positions (window_mode 0) or k_dev[f] near-equal runs
+ * (window_mode 1, see et_params).  k and w are clamped to [1, L]; a NaN score ranks below every
+ * number.  keep_dev bytes [N][L], count_dev int [N] = bytes set in each row. */
 ET_API et_status et_select_tokens(const float* scores_dev, const unsigned char* dynamic_dev, const int* k_dev,
-                           const int* w_dev, int N, int L, unsigned char* keep_dev, int* count_dev,
+                           const int* w_dev, int N, int L, int window_mode, unsigned char* keep_dev, int* count_dev,
                            void* cuda_stream);
 
 /* Paper Eq. 7: gather the kept rows of x_dev fp32 [N][L][D] in order into tokens_dev

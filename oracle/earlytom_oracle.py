@@ -304,19 +304,33 @@ def roles_of_segments(starts: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
 # Stage II: decoupled spatial token selection (Sec. 3.3, Algorithm 2)
 # ----------------------------------------------------------------------------------------------
 
-def rescaled_keep(r: float, B: int, N: int, L: int, retain_mode: int) -> Tuple[int, int, int]:
+def rescaled_keep(r: float, B: int, N: int, L: int, retain_mode: int, window_mode: int = 0) -> Tuple[int, int, int]:
     """Eq. 5-6.  The printed Eq. 5 cannot be used literally (it yields ~1e-3 where Eq. 6 needs a
     token amount), so r-hat is read as the per-frame token amount that restores the target ratio
     after Stage I removed B-N frames:  k = floor(r*B*L / N)  (mode 1) or floor(r*L) (mode 0),
-    clamped to [1, L];  window width w = floor(L / k) >= 1 and window count M = ceil(L / w)."""
+    clamped to [1, L];  window width w = floor(L / k) >= 1.
+    Window count M of a static frame: Eq. 6 as printed (window_mode 0) cuts windows of exactly w
+    positions, M = ceil(L / w), which is >= k and equals L as soon as k > L/2 (static frames then keep
+    every token and the target ratio is missed); window_mode 1 cuts M = k windows of near-equal width
+    (see `window_edges`), so that a static frame keeps exactly as many tokens as a dynamic one."""
     if retain_mode == 1:
         k = int(math.floor(r * B * L / N + 1e-9))
     else:
         k = int(math.floor(r * L + 1e-9))
     k = max(1, min(L, k))
     w = max(1, L // k)
-    M = -(-L // w)
+    M = k if window_mode == 1 else -(-L // w)
     return k, w, M
+
+
+def window_edges(L: int, k: int, w: int, window_mode: int = 0) -> List[int]:
+    """Boundaries e_0 = 0 < e_1 < ... < e_M = L of the local windows of a static frame (window m is
+    [e_m, e_{m+1})).  window_mode 0: Eq. 6 as printed, consecutive windows of w positions, the last one
+    possibly shorter.  window_mode 1: k windows with e_m = floor(m*L/k), widths floor(L/k) or that plus
+    one; identical to mode 0 whenever k divides L."""
+    if window_mode == 1:
+        return [(m * L) // k for m in range(k + 1)]
+    return list(range(0, L, w)) + [L]
 
 
 def topk_mask(a: np.ndarray, k: int) -> np.ndarray:
@@ -327,13 +341,14 @@ def topk_mask(a: np.ndarray, k: int) -> np.ndarray:
     return m
 
 
-def window_mask(a: np.ndarray, w: int) -> np.ndarray:
-    """Eq. 6: consecutive windows of width w over the flattened token index (last one may be
-    short); the maximum of each is kept, the lowest index among equals."""
+def window_mask(a: np.ndarray, w: int, k: int = 0, window_mode: int = 0) -> np.ndarray:
+    """Eq. 6: the maximum of each local window is kept, the lowest index among equals.  The windows
+    are those of `window_edges` (consecutive runs of w positions over the flattened token index in
+    mode 0, k near-equal runs in mode 1)."""
     L = len(a)
     m = np.zeros(L, dtype=bool)
-    for lo in range(0, L, w):
-        hi = min(lo + w, L)
+    edges = window_edges(L, k, w, window_mode)
+    for lo, hi in zip(edges[:-1], edges[1:]):
         best = lo
         for j in range(lo + 1, hi):
             if a[j] > a[best]:
@@ -370,7 +385,7 @@ def random_scores(seed: int, video: int, n_frames: int, L: int) -> np.ndarray:
     return (x >> np.uint32(8)).astype(np.float64) / float(1 << 24)
 
 
-def select_tokens(A: np.ndarray, dynamic: np.ndarray, k: int, w: int, selection: int) -> np.ndarray:
+def select_tokens(A: np.ndarray, dynamic: np.ndarray, k: int, w: int, selection: int, window_mode: int = 0) -> np.ndarray:
     """keep mask [N, L].  selection: 0 keep all, 1 decoupled (dynamic: top-k, static: windows),
     2 plain per-frame top-k on every frame (3, random sampling, is selection 2 applied to `random_scores`)."""
     N, L = A.shape
@@ -381,7 +396,7 @@ def select_tokens(A: np.ndarray, dynamic: np.ndarray, k: int, w: int, selection:
         elif selection == 2 or dynamic[f]:
             keep[f] = topk_mask(A[f], k)
         else:
-            keep[f] = window_mask(A[f], w)
+            keep[f] = window_mask(A[f], w, k, window_mode)
     return keep
 
 
@@ -440,21 +455,22 @@ def encode_video(frames: np.ndarray, shape, blob_or_w, params, dtype=np.float64,
     N = X.shape[0]
     feats = layer_norm(X, w["post_g"], w["post_b"], shape.ln_eps) if shape.post_layernorm else X
     if not merge_layers:
-        # Stage I is off: the segment list for Stage II comes from the streaming segmentation of
-        # the final features (Sec. 3.3: "similar to the streaming segmentation").
+        # Stage I is off: the segment list for Stage II comes from running the streaming segmentation
+        # of Sec. 3.2 on the final features (Sec. 3.3 says the division follows that segmentation).
         starts, _ = segment_by_similarity(frame_similarity(X), N, params.ema_alpha, params.tau_seg)
         sid, role = roles_of_segments(starts)
         for f in range(N):
             meta[f].seg_id, meta[f].role = int(sid[f]), int(role[f])
     dynamic = np.array([m.role != 1 for m in meta], dtype=bool)
-    k, wdt, M = rescaled_keep(params.retain, B, N, L, params.retain_mode)
+    wmode = int(getattr(params, "window_mode", 0))
+    k, wdt, M = rescaled_keep(params.retain, B, N, L, params.retain_mode, wmode)
     if forced is not None and "keep" in forced:
         keep = np.asarray(forced["keep"], dtype=bool)
     elif params.selection == 3:
         # random sampling (paper's sampling ablation): k tokens per frame, uniformly at random
         keep = select_tokens(random_scores(int(getattr(params, "sample_seed", 0)), video_index, N, L), dynamic, k, wdt, 2)
     else:
-        keep = select_tokens(A, dynamic, k, wdt, params.selection)
+        keep = select_tokens(A, dynamic, k, wdt, params.selection, wmode)
     counts = keep.sum(axis=1)
     offs = np.zeros(N + 1, dtype=np.int64)
     offs[1:] = np.cumsum(counts)

@@ -60,7 +60,8 @@ class et_params(C.Structure):
     _fields_ = [("num_merge_layers", C.c_int), ("merge_layers", C.c_int * ET_MAX_MERGE_LAYERS),
                 ("ema_alpha", C.c_double), ("tau_seg", C.c_double), ("tau_merge", C.c_double),
                 ("weighted_merge", C.c_int), ("selection", C.c_int), ("retain_mode", C.c_int), ("retain", C.c_double),
-                ("forced_plan", C.POINTER(et_forced_plan)), ("want_trace", C.c_int), ("sample_seed", C.c_ulonglong)]
+                ("forced_plan", C.POINTER(et_forced_plan)), ("want_trace", C.c_int), ("sample_seed", C.c_ulonglong),
+                ("window_mode", C.c_int)]
 
 
 class et_trace(C.Structure):
@@ -145,7 +146,7 @@ def load_library(path: str = _LIB_PATH) -> C.CDLL:
     lib.et_frame_similarity_static.argtypes = [vp, i, i, i, vp, vp]
     lib.et_merge_plan.argtypes = [vp, vp, i, i, d, d, d, i, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.et_merge_frames.argtypes = [vp, vp, i, i, vp, vp, vp, vp, vp, vp]
-    lib.et_select_tokens.argtypes = [vp, vp, vp, vp, i, i, vp, vp, vp]
+    lib.et_select_tokens.argtypes = [vp, vp, vp, vp, i, i, i, vp, vp, vp]
     lib.et_gather_tokens.argtypes = [vp, vp, i, i, i, vp, vp, f, vp, C.c_size_t, vp, vp, _I32P, vp]
     lib.et_linear_bf16.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, i, vp, vp]
     lib.et_attention.argtypes = [vp, vp, vp, i, i, i, i, i, vp]
@@ -269,6 +270,7 @@ def make_params(p, forced: Optional[ForcedPlan] = None, want_trace: bool = False
     q.retain = float(p.retain)
     q.want_trace = 1 if want_trace else 0
     q.sample_seed = int(getattr(p, "sample_seed", 0))
+    q.window_mode = int(getattr(p, "window_mode", 0))
     keep = []
     if forced is not None:
         fp = et_forced_plan()
@@ -492,12 +494,12 @@ def et_merge_frames(x, plan: dict, stream=None):
     return y
 
 
-def et_select_tokens(scores, dynamic, k, w, stream=None):
+def et_select_tokens(scores, dynamic, k, w, window_mode=0, stream=None):
     import torch
     N, L = scores.shape
     keep = torch.zeros((N, L), dtype=torch.uint8, device=scores.device)
     count = torch.zeros(N, dtype=torch.int32, device=scores.device)
-    _check(lib().et_select_tokens(_ptr(scores), _ptr(dynamic), _ptr(k), _ptr(w), N, L, _ptr(keep), _ptr(count),
+    _check(lib().et_select_tokens(_ptr(scores), _ptr(dynamic), _ptr(k), _ptr(w), N, L, int(window_mode), _ptr(keep), _ptr(count),
                                   _stream_ptr(stream)))
     return keep, count
 

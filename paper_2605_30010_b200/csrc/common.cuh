@@ -176,7 +176,7 @@ struct SelectSetupArgs {
 };
 void launch_select_setup(const SelectSetupArgs& a, int n_cap, cudaStream_t s);
 void launch_select_tokens(const float* scores, const unsigned char* dynamic, const int* k_frame, const int* w_frame,
-                          int n_cap, int L, int selection_all, unsigned char* keep, int* count,
+                          int n_cap, int L, int selection_all, int window_mode, unsigned char* keep, int* count,
                           const int* n_frames_dev, cudaStream_t s);
 // Random-sampling ablation: scores[f][j] = uniform number of Philox-4x32-10 with counter (j, frame inside its
 // video, video, 0) and key = seed, for the frames of the current list.

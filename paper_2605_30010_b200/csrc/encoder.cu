@@ -188,6 +188,7 @@ et_status validate_config(const et_config* c) {
   if (c->dtype != ET_F32 && c->dtype != ET_BF16) return ET_ERR_INVALID_ARG;
   if (c->dtype == ET_BF16 && (c->hidden % 8 != 0 || c->mlp_dim % 8 != 0 || (c->hidden / c->heads) % 8 != 0)) return ET_ERR_SHAPE;
   if (c->max_frames_total < 1 || c->max_videos < 1 || c->max_videos > 1024) return ET_ERR_INVALID_ARG;
+  if (c->max_frames_total > 65535) return ET_ERR_CAPACITY;      // frames index gridDim.y of the merge and gather kernels
   const long long L = (long long)(c->image_size / c->patch_size) * (c->image_size / c->patch_size);
   if (L > 4096 || L * c->max_frames_total > (1ll << 30)) return ET_ERR_CAPACITY;
   if (!(c->ln_eps > 0.f)) return ET_ERR_INVALID_ARG;
@@ -206,6 +207,7 @@ et_status validate_params(const et_encoder* e, const et_params* p) {
   if (isnan(p->tau_seg) || isnan(p->tau_merge)) return ET_ERR_INVALID_ARG;
   if (p->selection < 0 || p->selection > 3) return ET_ERR_INVALID_ARG;
   if (p->retain_mode < 0 || p->retain_mode > 1) return ET_ERR_INVALID_ARG;
+  if (p->window_mode < 0 || p->window_mode > 1) return ET_ERR_INVALID_ARG;
   return ET_OK;
 }
 
@@ -349,7 +351,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
       sel_scores = e->score_partial;
     }
     if (rank_all) ET_CUDA(e, cudaMemsetAsync(e->dynamic, 1, T, s));            // every frame ranks globally
-    PROF(ET_CAT_SELECT, launch_select_tokens(sel_scores, e->dynamic, e->k_frame, e->w_frame, T, L, p->selection == 0, e->keep, e->count, n_dev, s));
+    PROF(ET_CAT_SELECT, launch_select_tokens(sel_scores, e->dynamic, e->k_frame, e->w_frame, T, L, p->selection == 0, p->window_mode, e->keep, e->count, n_dev, s));
     if (rank_all) PROF(ET_CAT_SELECT, launch_select_setup(sa, T, s));          // restore the reported dynamic flags
   }
   PROF(ET_CAT_SELECT, launch_scan_counts(e->count, e->frame_offsets, e->d_small, T, n_dev, s));
@@ -707,10 +709,12 @@ et_status et_merge_frames(const float* x_dev, float* y_dev, int n_cap, int frame
 }
 
 et_status et_select_tokens(const float* scores_dev, const unsigned char* dynamic_dev, const int* k_dev, const int* w_dev,
-                           int N, int L, unsigned char* keep_dev, int* count_dev, void* cuda_stream) {
+                           int N, int L, int window_mode, unsigned char* keep_dev, int* count_dev, void* cuda_stream) {
   if (!scores_dev || !dynamic_dev || !k_dev || !w_dev || !keep_dev || !count_dev) return ET_ERR_INVALID_ARG;
+  if (window_mode < 0 || window_mode > 1) return ET_ERR_INVALID_ARG;
   if (N < 1 || L < 1 || L > 4096) return ET_ERR_SHAPE;
-  launch_select_tokens(scores_dev, dynamic_dev, k_dev, w_dev, N, L, 0, keep_dev, count_dev, nullptr, (cudaStream_t)cuda_stream);
+  launch_select_tokens(scores_dev, dynamic_dev, k_dev, w_dev, N, L, 0, window_mode, keep_dev, count_dev, nullptr,
+                       (cudaStream_t)cuda_stream);
   ET_CUDA0(cudaGetLastError());
   return ET_OK;
 }

@@ -19,7 +19,7 @@ __global__ void select_setup_kernel(SelectSetupArgs a) {
     if (a.retain_mode == 1) k = (int)floor(a.retain * (double)B * (double)a.L / (double)max(N, 1) + 1e-9);
     else k = (int)floor(a.retain * (double)a.L + 1e-9);
     k = max(1, min(a.L, k));
-    const int w = max(1, a.L / k);
+    const int w = max(1, a.L / k);      // reported in both window modes; mode 1 cuts k near-equal windows instead
     a.video_k[v] = k;
     a.video_w[v] = w;
   }
@@ -45,12 +45,18 @@ void launch_select_setup(const SelectSetupArgs& a, int n_cap, cudaStream_t s) {
 // Selection: one CTA per frame, scores in shared memory.
 //   dynamic frame: token j is kept iff fewer than k tokens precede it in the order
 //                  (score descending, index ascending)  -> exact rank counting, O(L^2 / threads);
-//   static frame : the first maximum of each window of width w.
+//   static frame : the first maximum of each window; windows are runs of w positions (window_mode 0,
+//                  Eq. 6 as printed) or the k runs [floor(m L / k), floor((m+1) L / k)) (window_mode 1).
+// A NaN score compares false against everything: it is ordered as the lowest value (after every number,
+// ties to the lower index), so a frame never keeps more than k tokens and count[f] is the number of
+// bytes set in the mask.  k and w are clamped to [1, L].
 // ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float nan_to_lowest(float v) { return v != v ? -INFINITY : v; }
+
 __global__ void __launch_bounds__(256)
 select_tokens_kernel(const float* __restrict__ scores, const unsigned char* __restrict__ dynamic,
                      const int* __restrict__ k_frame, const int* __restrict__ w_frame, int n_cap, int L,
-                     int selection_all, unsigned char* __restrict__ keep, int* __restrict__ count,
+                     int selection_all, int window_mode, unsigned char* __restrict__ keep, int* __restrict__ count,
                      const int* __restrict__ n_frames_dev) {
   extern __shared__ float sh_a[];
   const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
@@ -63,10 +69,10 @@ select_tokens_kernel(const float* __restrict__ scores, const unsigned char* __re
     if (threadIdx.x == 0) count[f] = L;
     return;
   }
-  for (int j = threadIdx.x; j < L; j += blockDim.x) sh_a[j] = a[j];
+  for (int j = threadIdx.x; j < L; j += blockDim.x) sh_a[j] = nan_to_lowest(a[j]);
   __syncthreads();
+  const int k = max(1, min(k_frame[f], L));
   if (dynamic[f]) {
-    const int k = k_frame[f];
     for (int j = threadIdx.x; j < L; j += blockDim.x) {
       const float aj = sh_a[j];
       int rank = 0;
@@ -76,30 +82,31 @@ select_tokens_kernel(const float* __restrict__ scores, const unsigned char* __re
       }
       kp[j] = rank < k ? 1 : 0;
     }
-    if (threadIdx.x == 0) count[f] = min(k, L);
+    if (threadIdx.x == 0) count[f] = k;       // the order is total, so exactly k ranks are below k
   } else {
-    const int w = w_frame[f];
-    const int M = (L + w - 1) / w;
+    const int w = max(1, min(w_frame[f], L));
+    const int M = window_mode == 1 ? k : (L + w - 1) / w;
     for (int j = threadIdx.x; j < L; j += blockDim.x) kp[j] = 0;
     __syncthreads();
     for (int m = threadIdx.x; m < M; m += blockDim.x) {
-      const int lo = m * w, hi = min(lo + w, L);
+      const int lo = window_mode == 1 ? (int)(((long long)m * L) / k) : m * w;
+      const int hi = window_mode == 1 ? (int)(((long long)(m + 1) * L) / k) : min(lo + w, L);
       int best = lo;
       for (int j = lo + 1; j < hi; ++j)
         if (sh_a[j] > sh_a[best]) best = j;
       kp[best] = 1;
     }
-    if (threadIdx.x == 0) count[f] = M;
+    if (threadIdx.x == 0) count[f] = M;       // windows are disjoint and non-empty: one byte set per window
   }
 }
 
 void launch_select_tokens(const float* scores, const unsigned char* dynamic, const int* k_frame, const int* w_frame,
-                          int n_cap, int L, int selection_all, unsigned char* keep, int* count,
+                          int n_cap, int L, int selection_all, int window_mode, unsigned char* keep, int* count,
                           const int* n_frames_dev, cudaStream_t s) {
   if (n_cap <= 0) return;
   ET_COUNT_LAUNCH();
   select_tokens_kernel<<<n_cap, 256, sizeof(float) * L, s>>>(scores, dynamic, k_frame, w_frame, n_cap, L,
-                                                             selection_all, keep, count, n_frames_dev);
+                                                             selection_all, window_mode, keep, count, n_frames_dev);
 }
 
 // ---------------------------------------------------------------------------------------------

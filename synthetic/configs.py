@@ -61,6 +61,7 @@ class MergeParams:
     retain_mode: int = 1    # 0 per-frame fraction, 1 total budget
     retain: float = 0.25
     sample_seed: int = 0    # seed of the random-sampling ablation (selection 3)
+    window_mode: int = 1    # static frames: 0 = windows of floor(L/k) positions (Eq. 6 as printed), 1 = k near-equal windows
 
 
 @dataclass(frozen=True)

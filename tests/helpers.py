@@ -66,7 +66,16 @@ def compare_stage1(gpu_trace, oracle_results, params, sim_tol, log):
     return True
 
 
-def compare_keep(gpu_keep, gpu_scores, ora_keep, ora_scores, dynamic, k, w, score_tol, log):
+def window_of(j, L, k, w, window_mode):
+    """[lo, hi) of the local window position j of a static frame falls into."""
+    if window_mode == 1:
+        m = -(-((j + 1) * k) // L) - 1
+        return (m * L) // k, ((m + 1) * L) // k
+    lo = (j // w) * w
+    return lo, min(lo + w, L)
+
+
+def compare_keep(gpu_keep, gpu_scores, ora_keep, ora_scores, dynamic, k, w, score_tol, log, window_mode=0):
     """Kept sets must be equal except where the oracle's score is within the near-tie band of the
     cut (k-th score on dynamic frames, the window's maximum on static frames)."""
     N, L = ora_keep.shape
@@ -86,8 +95,8 @@ def compare_keep(gpu_keep, gpu_scores, ora_keep, ora_scores, dynamic, k, w, scor
                 log.append(f"near-tie: frame {f} token {j} top-k, rel margin {rel:.2e}")
         else:
             for j in diff:
-                lo = (j // w) * w
-                win = a[lo:lo + w]
+                lo, hi = window_of(int(j), L, k, w, window_mode)
+                win = a[lo:hi]
                 rel = abs(a[j] - win.max()) / abs(win.max())
                 if rel > SCORE_TIE + score_tol:
                     raise AssertionError(f"frame {f} token {j}: window argmax differs, rel margin {rel:.3e}")

@@ -59,7 +59,7 @@ def check_against_oracle(B, enc, frames, offs, params, results, tol, sim_tol, sc
         if params.selection != 0:
             dynv = r.frame_dynamic if params.selection == 1 else np.ones(N, dtype=bool)
             keep_same &= H.compare_keep(run.trace.keep[f0:f0 + N], run.trace.scores[f0:f0 + N], r.keep, r.scores,
-                                        dynv, r.k, r.w, score_tol, log)
+                                        dynv, r.k, r.w, score_tol, log, params.window_mode)
         f0 += N
     final = run if (stage1_same and keep_same) else enc.encode_batch(fr, offs, params, want_trace=True,
                                                                       forced=B.ForcedPlan(seg, mrg, keep))

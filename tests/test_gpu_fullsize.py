@@ -77,9 +77,9 @@ def _check_decisions(run, wl, offs):
     for v in range(len(cur) - 1):
         f0, f1 = int(cur[v]), int(cur[v + 1])
         Bv = int(offs[v + 1] - offs[v])
-        k, w, M = O.rescaled_keep(p.retain, Bv, f1 - f0, L, p.retain_mode)
+        k, w, M = O.rescaled_keep(p.retain, Bv, f1 - f0, L, p.retain_mode, p.window_mode)
         assert tr.video_k[v] == k and tr.video_w[v] == w
-        keep = O.select_tokens(tr.scores[f0:f1].astype(np.float64), run["dynamic"][f0:f1], k, w, p.selection)
+        keep = O.select_tokens(tr.scores[f0:f1].astype(np.float64), run["dynamic"][f0:f1], k, w, p.selection, p.window_mode)
         np.testing.assert_array_equal(tr.keep[f0:f1].astype(bool), keep, err_msg=f"video {v} kept set")
         np.testing.assert_allclose(tr.scores[f0:f1].sum(axis=1), 1.0, atol=2e-3)
     return cur

@@ -117,21 +117,47 @@ def test_merge_frames_matches_eq3(B):
 
 # ------------------------------------------------------------------ Stage II
 
-@pytest.mark.parametrize("N,L", [(6, 64), (3, 729), (4, 17), (1, 1)])
-def test_select_tokens_exact(B, N, L):
+@pytest.mark.parametrize("window_mode", [0, 1])
+@pytest.mark.parametrize("N,L", [(6, 64), (3, 729), (4, 17), (1, 1), (40, 729)])
+def test_select_tokens_exact(B, N, L, window_mode):
     rng = np.random.default_rng(N * 100 + L)
     a = rng.random((N, L)).astype(np.float32)
     a[:, ::3] = np.round(a[:, ::3] * 4) / 4          # exact ties
     dyn = (rng.random(N) < 0.5).astype(np.uint8)
     dyn[0] = 1
     k = rng.integers(1, L + 1, N).astype(np.int32)
+    if N > 2:
+        k[1], k[2] = L, 1                            # the extremes: keep everything / one token
     w = np.maximum(1, L // k).astype(np.int32)
-    keep, count = B.et_select_tokens(cuda(a), cuda(dyn), cuda(k), cuda(w))
+    keep, count = B.et_select_tokens(cuda(a), cuda(dyn), cuda(k), cuda(w), window_mode)
     keep = keep.cpu().numpy().astype(bool)
     for f in range(N):
-        ref = O.topk_mask(a[f], int(k[f])) if dyn[f] else O.window_mask(a[f], int(w[f]))
+        ref = O.topk_mask(a[f], int(k[f])) if dyn[f] else O.window_mask(a[f], int(w[f]), int(k[f]), window_mode)
         np.testing.assert_array_equal(keep[f], ref)
         assert int(count[f].item()) == ref.sum()
+
+
+def test_select_tokens_degenerate_inputs(B):
+    """Out-of-range amounts are clamped to [1, L]; a NaN score ranks below every number, so the kept count never
+    exceeds k and count[] always equals the bytes set in the mask (what the gather's offsets rely on)."""
+    L = 50
+    rng = np.random.default_rng(0)
+    a = rng.random((4, L)).astype(np.float32)
+    a[0, [3, 7, 20]] = np.nan
+    a[1, :] = np.nan
+    dyn = np.array([1, 1, 0, 0], dtype=np.uint8)
+    k = np.array([10, 5, 0, 99], dtype=np.int32)
+    w = np.array([5, 10, 0, -3], dtype=np.int32)
+    for mode in (0, 1):
+        keep, count = B.et_select_tokens(cuda(a), cuda(dyn), cuda(k), cuda(w), mode)
+        keep = keep.cpu().numpy().astype(bool)
+        np.testing.assert_array_equal(keep.sum(axis=1), count.cpu().numpy())
+        finite = np.where(np.isnan(a[0]), -np.inf, a[0])
+        np.testing.assert_array_equal(keep[0], O.topk_mask(finite, 10))
+        assert not keep[0, [3, 7, 20]].any()
+        assert np.nonzero(keep[1])[0].tolist() == [0, 1, 2, 3, 4]     # all equal: lowest indices
+        assert count[2].item() == (1 if mode == 1 else L)              # k = 0 -> 1 ; w = 0 -> 1
+        assert count[3].item() == L                                    # k = 99 -> L ; w < 1 -> 1
 
 
 @pytest.mark.parametrize("N,L,D,ln", [(5, 64, 64, True), (3, 729, 1152, True), (4, 30, 12, False), (2, 100, 2048, True)])

@@ -190,6 +190,70 @@ def test_eq3_golden_weights():
     np.testing.assert_allclose(m, 1.5, atol=1e-12)
 
 
+def _rotated_frames(angles, L=6, D=8, seed=0):
+    """Frames whose token at every position is r_l * (cos(theta_t) e1 + sin(theta_t) e2) for a fixed orthonormal
+    pair (e1, e2) and positive per-position lengths r_l (differing between frames): the cosine of every position of
+    frames t, t+1 is cos(theta_{t+1} - theta_t), hence so is their similarity -- known without running any code."""
+    rng = np.random.default_rng(seed)
+    q, _ = np.linalg.qr(rng.standard_normal((D, 2)))
+    e1, e2 = q[:, 0], q[:, 1]
+    frames = []
+    for th in angles:
+        r = rng.uniform(0.5, 2.0, size=(L, 1))
+        frames.append(r * (np.cos(th) * e1 + np.sin(th) * e2)[None, :])
+    return np.stack(frames)
+
+
+def test_assembled_step_uses_similarity_to_the_following_frame_as_eq3_weights():
+    """One segment [H, X, Y, Z, T] with similarities c = cos(.3), cos(.2), cos(.5), cos(.1).  Eq. 2 picks the pair
+    (X, Y) (c_1 > tau and c_1 > c_2); Eq. 3 then weights X by c_1 = Sim(X, Y) and Y by c_2 = Sim(Y, Z): each frame by
+    its similarity with the frame after it.  A step that took (c_0, c_1) or (c_1, c_3) instead gives other weights."""
+    import math
+    th = np.cumsum([0.0, 0.3, 0.2, 0.5, 0.1])
+    F = _rotated_frames(th)
+    c = [math.cos(0.3), math.cos(0.2), math.cos(0.5), math.cos(0.1)]
+    wa, wb = c[1] / (c[1] + c[2]), c[2] / (c[1] + c[2])
+    expect = wa * F[1] + wb * F[2]
+    meta = [O.FrameMeta(t, t) for t in range(5)]
+    for run in ("free", "forced"):
+        if run == "free":
+            Fo, mo, tr = O.stage1_one_video(F, meta, 0.9, -2.0, 0.5, True, 0)
+        else:
+            decision = (np.array([1, 0, 0, 0, 0], bool), np.array([0, 1, 0, 0, 0], bool))
+            Fo, mo, tr = O._stage1_forced(F, meta, decision, True, 0)
+        np.testing.assert_allclose(tr.c, c, atol=1e-12)
+        assert np.nonzero(tr.merge_with_next)[0].tolist() == [1] and tr.n_out == 4
+        np.testing.assert_allclose(tr.w_a, [1.0, wa, 1.0, 1.0], atol=1e-12)
+        np.testing.assert_allclose(tr.w_b, [0.0, wb, 0.0, 0.0], atol=1e-12)
+        assert tr.src_a.tolist() == [0, 1, 3, 4] and tr.src_b.tolist() == [-1, 2, -1, -1]
+        np.testing.assert_allclose(Fo[1], expect, atol=1e-12)
+        np.testing.assert_array_equal(Fo[[0, 2, 3]], F[[0, 3, 4]])
+        # the plausible wrong choices are far outside the tolerance
+        for sa, sb in ((c[0], c[1]), (c[1], c[3]), (c[2], c[1])):
+            wrong = (sa * F[1] + sb * F[2]) / (sa + sb)
+            assert np.abs(wrong - expect).max() > 1e-3
+    # unweighted variant: plain mean, whatever the similarities
+    Fo, _, tr = O.stage1_one_video(F, meta, 0.9, -2.0, 0.5, False, 0)
+    np.testing.assert_allclose(Fo[1], 0.5 * (F[1] + F[2]), atol=1e-12)
+    np.testing.assert_allclose(tr.w_a[1], 0.5)
+
+
+def test_assembled_step_two_pairs_and_later_layer():
+    """Seven frames, decreasing similarities inside one segment: pairs (1,2) and (3,4) merge, each with its own two
+    similarities; a second pass over the merged list (the way several merge layers compose) uses the similarities of
+    the merged list, again known in closed form because a merged frame stays in the (e1, e2) plane."""
+    import math
+    d = [0.10, 0.15, 0.20, 0.25, 0.30, 0.05]
+    th = np.cumsum([0.0] + d)
+    F = _rotated_frames(th, seed=3)
+    c = [math.cos(x) for x in d]
+    Fo, mo, tr = O.stage1_one_video(F, [O.FrameMeta(t, t) for t in range(7)], 0.9, -2.0, 0.5, True, 0)
+    assert np.nonzero(tr.merge_with_next)[0].tolist() == [1, 3]
+    np.testing.assert_allclose(Fo[1], (c[1] * F[1] + c[2] * F[2]) / (c[1] + c[2]), atol=1e-12)
+    np.testing.assert_allclose(Fo[2], (c[3] * F[3] + c[4] * F[4]) / (c[3] + c[4]), atol=1e-12)
+    assert [(m.src_lo, m.src_hi) for m in mo] == [(0, 0), (1, 2), (3, 4), (5, 5), (6, 6)]
+
+
 def test_identical_middle_pair_collapses():
     """[H, X, X, Y, T] in one segment: the two X have similarity 1 > the next similarity, so they
     merge into one frame equal to X; every other frame is copied."""

@@ -62,6 +62,40 @@ def test_window_bruteforce():
             assert np.nonzero(m[lo:lo + w])[0][0] == int(np.argmax(win))   # first maximum
 
 
+def test_balanced_windows_closed_form_and_budget():
+    """window_mode 1: k windows [floor(m L / k), floor((m+1) L / k)).  Pinned by the closed form of the window
+    a position falls into, m(j) = ceil((j+1) k / L) - 1, which never uses the edges; by the widths; by equality
+    with Eq. 6 as printed whenever k divides L; and by the kept total N*k against the budget r*B*L."""
+    rng = np.random.default_rng(11)
+    for trial in range(300):
+        L = int(rng.integers(1, 40))
+        k = int(rng.integers(1, L + 1))
+        w = L // k
+        e = O.window_edges(L, k, w, 1)
+        assert e[0] == 0 and e[-1] == L and len(e) == k + 1
+        widths = np.diff(e)
+        assert widths.min() >= 1 and set(widths.tolist()) <= {w, w + 1}
+        a = rng.integers(0, 4, L).astype(np.float64)
+        m = O.window_mask(a, w, k, 1)
+        assert m.sum() == k
+        win_of = [-(-((j + 1) * k) // L) - 1 for j in range(L)]
+        for mm in range(k):
+            members = [j for j in range(L) if win_of[j] == mm]
+            best = max(members, key=lambda j: (a[j], -j))                   # first maximum
+            assert m[members].sum() == 1 and m[best]
+        if L % k == 0:
+            assert e == O.window_edges(L, k, w, 0)
+            np.testing.assert_array_equal(m, O.window_mask(a, w))
+    # the budget: static and dynamic frames both keep k, so the total is N*k, within N of r*B*L
+    for B, N, L, r in [(32, 13, 729, 0.25), (32, 24, 729, 0.25), (32, 12, 729, 0.10), (64, 40, 729, 0.25)]:
+        k, w, M = O.rescaled_keep(r, B, N, L, 1, window_mode=1)
+        assert M == k and abs(N * k - r * B * L) < N
+    # Eq. 6 as printed misses it as soon as k > L/2: every static frame keeps all L tokens
+    k, w, M = O.rescaled_keep(0.25, 32, 13, 729, 1, window_mode=0)
+    assert (k, w, M) == (448, 1, 729)
+    assert O.rescaled_keep(0.25, 32, 13, 729, 1, window_mode=1) == (448, 1, 448)
+
+
 def test_selection_counts_and_roles():
     rng = np.random.default_rng(2)
     A = rng.random((5, 16))
@@ -70,6 +104,7 @@ def test_selection_counts_and_roles():
     assert keep.sum(axis=1).tolist() == [4, 4, 4, 4, 4]
     keep = O.select_tokens(A, dyn, 5, 3, 1)          # w = 16 // 5 = 3 -> M = 6 windows on static frames
     assert keep.sum(axis=1).tolist() == [5, 6, 6, 5, 5]
+    assert O.select_tokens(A, dyn, 5, 3, 1, window_mode=1).sum(axis=1).tolist() == [5] * 5
     assert O.select_tokens(A, dyn, 5, 3, 2).sum(axis=1).tolist() == [5] * 5
     assert O.select_tokens(A, dyn, 5, 3, 0).all()
 
@@ -110,7 +145,7 @@ def test_end_to_end_bookkeeping():
     # dynamic = head/tail of the segments of the last merge layer
     T = int(r.frame_dynamic.sum())
     assert r.tokens.shape[0] == T * r.k + (N - T) * r.M
-    assert (r.k, r.w, r.M) == O.rescaled_keep(p.retain, B, N, L, 1)
+    assert (r.k, r.w, r.M) == O.rescaled_keep(p.retain, B, N, L, 1, p.window_mode)
     assert r.frame_src_lo[0] == 0 and r.frame_src_hi[-1] == B - 1
     assert (r.frame_src_hi[:-1] + 1 == r.frame_src_lo[1:]).all()
 
