@@ -292,7 +292,7 @@ def main():
     n_rot = 4 if V == 1 else 2
     sets = []
     for sd in rank_video_seeds(rank, n_rot):
-        vs = [make_video(v.n_frames, shape.image_size, shape.patch_size, v.resample_p, v.seed + sd, v.jitter) for v in wl.videos]
+        vs = [make_video(v.n_frames, shape.image_size, shape.patch_size, v.resample_p, v.seed + sd, v.jitter, v.cut_every) for v in wl.videos]
         sets.append(np.ascontiguousarray(np.concatenate(vs, axis=0)))
     vids = sets
     offs = [0]

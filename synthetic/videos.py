@@ -6,7 +6,9 @@ channel, bilinearly interpolated); every following frame copies its predecessor
 and replaces exactly round(p * P) of the P = (H // patch)**2 patches by fresh
 smooth noise.  An optional per-frame global brightness offset, uniform in
 [-jitter, +jitter], is added to that frame only (it does not accumulate).
-Pixels are finally mapped from [0, 1] to [-1, 1].  Output: float32 [T, 3, H, W].
+With cut_every = c > 0 every c-th frame (t = c, 2c, ...) is a scene cut: all of its
+patches are fresh, so the similarity to its predecessor drops to that of unrelated
+images.  Pixels are finally mapped from [0, 1] to [-1, 1].  Output: float32 [T, 3, H, W].
 """
 from __future__ import annotations
 
@@ -32,7 +34,7 @@ def _smooth_field(rng: np.random.Generator, size: int) -> np.ndarray:
 
 
 def make_video(n_frames: int, image_size: int, patch_size: int, resample_p: float,
-               seed: int, jitter: float = 0.0) -> np.ndarray:
+               seed: int, jitter: float = 0.0, cut_every: int = 0) -> np.ndarray:
     grid = image_size // patch_size
     n_patches = grid * grid
     n_swap = int(round(resample_p * n_patches))
@@ -41,9 +43,10 @@ def make_video(n_frames: int, image_size: int, patch_size: int, resample_p: floa
     jit = _rng(seed, 2)
     frames = np.empty((n_frames, 3, image_size, image_size), dtype=np.float32)
     for t in range(n_frames):
-        if t > 0 and n_swap > 0:
+        cut = cut_every > 0 and t > 0 and t % cut_every == 0
+        if t > 0 and (n_swap > 0 or cut):
             fresh = _smooth_field(_rng(seed, 16 + t), image_size)
-            chosen = pick.permutation(n_patches)[:n_swap]
+            chosen = pick.permutation(n_patches)[:n_patches if cut else n_swap]
             for pidx in chosen:
                 y0 = (int(pidx) // grid) * patch_size
                 x0 = (int(pidx) % grid) * patch_size
@@ -57,7 +60,7 @@ def make_video(n_frames: int, image_size: int, patch_size: int, resample_p: floa
 def make_batch(workload) -> tuple[np.ndarray, np.ndarray]:
     """All videos of a workload concatenated along the frame axis, plus int32 offsets [V+1]."""
     s = workload.shape
-    vids = [make_video(v.n_frames, s.image_size, s.patch_size, v.resample_p, v.seed, v.jitter)
+    vids = [make_video(v.n_frames, s.image_size, s.patch_size, v.resample_p, v.seed, v.jitter, v.cut_every)
             for v in workload.videos]
     offs = np.zeros(len(vids) + 1, dtype=np.int32)
     offs[1:] = np.cumsum([v.shape[0] for v in vids])

@@ -27,63 +27,17 @@ def to_cuda(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def oracle_forced(results):
-    """Oracle decisions of all videos, concatenated in the layout the library's forced plan uses."""
-    nm = len(results[0].merge_trace)
-    seg = [np.concatenate([r.merge_trace[i].starts for r in results]) for i in range(nm)]
-    mrg = [np.concatenate([r.merge_trace[i].merge_with_next for r in results]) for i in range(nm)]
-    keep = np.concatenate([r.keep for r in results], axis=0)
-    return seg, mrg, keep
+# Hard ceilings on the numeric error of the decision quantities (the near-tie band itself is widened by the error
+# MEASURED in the run, see tests/helpers.py).  Measured on B200: fp32 path similarity error <= 7e-8, score error
+# <= 4e-7 of the largest score (rounding order only); bf16 path similarity error <= 7.2e-5 (the cosines come from
+# the fp32 residual stream and the errors of 729 positions average out), score error <= 3.5e-3 of the largest
+# score.  The ceilings are those figures times 7 (similarity) and 3 (scores), rounded.
+F32_SIM, F32_SCORE = 1e-6, 5e-6
+BF16_SIM, BF16_SCORE = 5e-4, 1e-2
+NEAR_TIE_SHARE = 0.005       # at most 0.5 % of the decisions of a workload may be logged near-ties (measured: <= 0.2 %)
 
 
-def check_against_oracle(B, enc, frames, offs, params, results, tol, sim_tol, score_tol):
-    """The comparison protocol: decisions first (near-ties logged), then values under identical decisions."""
-    log = []
-    fr = to_cuda(frames)
-    free = enc.encode_batch(fr, offs, params, want_trace=True)
-    seg, mrg, keep = oracle_forced(results)
-    stage1_same = H.compare_stage1(free.trace, results, params, sim_tol, log) if params.merge_layers else True
-    run = free if stage1_same else enc.encode_batch(fr, offs, params, want_trace=True,
-                                                    forced=B.ForcedPlan(seg, mrg, None))
-    # Stage II decisions under identical Stage I decisions
-    ora_scores = np.concatenate([r.scores for r in results], axis=0)
-    dyn = np.concatenate([r.frame_dynamic for r in results])
-    np.testing.assert_array_equal(run.frame_dynamic.cpu().numpy().astype(bool), dyn)
-    rel = np.abs(run.trace.scores - ora_scores).max() / ora_scores.max()
-    assert rel <= score_tol, f"attention scores differ by {rel:.3e} of the maximum"
-    f0 = 0
-    keep_same = True
-    for v, r in enumerate(results):
-        N = len(r.frame_dynamic)
-        assert run.trace.video_k[v] == r.k and run.trace.video_w[v] == r.w
-        if params.selection != 0:
-            dynv = r.frame_dynamic if params.selection == 1 else np.ones(N, dtype=bool)
-            keep_same &= H.compare_keep(run.trace.keep[f0:f0 + N], run.trace.scores[f0:f0 + N], r.keep, r.scores,
-                                        dynv, r.k, r.w, score_tol, log, params.window_mode)
-        f0 += N
-    final = run if (stage1_same and keep_same) else enc.encode_batch(fr, offs, params, want_trace=True,
-                                                                      forced=B.ForcedPlan(seg, mrg, keep))
-    # values and index map under identical decisions
-    toks = np.concatenate([r.tokens for r in results], axis=0)
-    assert final.n_tokens == toks.shape[0]
-    err = H.token_error(final.tokens.cpu().numpy(), toks)
-    assert err <= tol, f"token error {err:.3e} > {tol}"
-    np.testing.assert_array_equal(final.token_pos.cpu().numpy(), np.concatenate([r.token_pos for r in results]))
-    fo = [0]
-    for r in results:
-        fo += list(fo[-1] + r.frame_offsets[1:])
-    np.testing.assert_array_equal(final.frame_offsets.cpu().numpy(), np.array(fo))
-    np.testing.assert_array_equal(final.frame_src_lo.cpu().numpy(), np.concatenate([r.frame_src_lo for r in results]))
-    np.testing.assert_array_equal(final.frame_src_hi.cpu().numpy(), np.concatenate([r.frame_src_hi for r in results]))
-    vfo = np.concatenate([[0], np.cumsum([len(r.frame_dynamic) for r in results])])
-    np.testing.assert_array_equal(final.video_frame_offsets.cpu().numpy(), vfo)
-    assert final.frames_per_block == [sum(r.frames_per_block[i] for r in results) for i in range(len(final.frames_per_block))]
-    for line in log:
-        print(line)
-    return err, log
-
-
-def run_workload(B, wl, oracle_dtype, tol, sim_tol, score_tol, params=None):
+def run_workload(B, wl, oracle_dtype, tol, sim_ceiling, score_ceiling, params=None):
     params = params or wl.params
     frames, offs = make_batch(wl)
     blob = make_weights(wl.shape, wl.weight_seed, wl.pos_std)
@@ -91,34 +45,37 @@ def run_workload(B, wl, oracle_dtype, tol, sim_tol, score_tol, params=None):
     results = O.encode_batch(frames, offs, wl.shape, w, params, dtype=oracle_dtype)
     enc = B.Encoder(wl.shape, blob, B.ET_F32 if wl.dtype == "f32" else B.ET_BF16, wl.total_frames, len(wl.videos))
     try:
-        return check_against_oracle(B, enc, frames, offs, params, results, tol, sim_tol, score_tol)
+        stats, log = H.check_parity(B, enc, to_cuda(frames), offs, params, H.batch_from_results(results), tol,
+                                    sim_ceiling, score_ceiling, wl.name)
     finally:
         enc.close()
+    assert stats["near_ties"] <= max(1, NEAR_TIE_SHARE * stats["decisions"]), stats
+    return stats["token_err"], log
 
 
 # ------------------------------------------------------------------ fp32 path
 
 def test_tiny_fp32_workload(B):
-    err, log = run_workload(B, workload("tiny"), np.float64, F32_TOL, 1e-5, 1e-4)
+    err, log = run_workload(B, workload("tiny"), np.float64, F32_TOL, F32_SIM, F32_SCORE)
     assert not log, "no near-tie expected on the fp32 tiny workload"
 
 
 def test_tiny_fp32_uncompressed(B):
     wl = workload("tiny").uncompressed()
-    run_workload(B, wl, np.float64, F32_TOL, 1e-5, 1e-4)
+    run_workload(B, wl, np.float64, F32_TOL, F32_SIM, F32_SCORE)
 
 
 @pytest.mark.parametrize("selection,mode,retain", [(2, 0, 0.25), (1, 1, 0.3), (0, 1, 1.0), (3, 0, 0.25)])
 def test_tiny_fp32_variants(B, selection, mode, retain):
     wl = workload("tiny")
     p = dataclasses.replace(wl.params, selection=selection, retain_mode=mode, retain=retain, tau_seg=0.895, tau_merge=0.85)
-    run_workload(B, wl, np.float64, F32_TOL, 1e-5, 1e-4, params=p)
+    run_workload(B, wl, np.float64, F32_TOL, F32_SIM, F32_SCORE, params=p)
 
 
 def test_tiny_fp32_unweighted_merge_and_erf_gelu(B):
     wl = workload("tiny")
     wl = dataclasses.replace(wl, shape=dataclasses.replace(wl.shape, gelu_tanh=0, post_layernorm=0))
-    run_workload(B, wl, np.float64, F32_TOL, 1e-5, 1e-4, params=dataclasses.replace(wl.params, weighted_merge=0))
+    run_workload(B, wl, np.float64, F32_TOL, F32_SIM, F32_SCORE, params=dataclasses.replace(wl.params, weighted_merge=0))
 
 
 def test_fp32_batch_of_ragged_videos(B):
@@ -126,7 +83,7 @@ def test_fp32_batch_of_ragged_videos(B):
     vids = (VideoSpec(5, 0.1, 1), VideoSpec(1, 0.2, 2), VideoSpec(9, 0.05, 3), VideoSpec(2, 0.5, 4), VideoSpec(12, 0.15, 5))
     p = MergeParams(merge_layers=(1, 3), tau_seg=0.6, tau_merge=0.7, selection=1, retain_mode=1, retain=0.4)
     wl = Workload("ragged", shape, "f32", vids, p, 77)
-    run_workload(B, wl, np.float64, F32_TOL, 1e-5, 1e-4)
+    run_workload(B, wl, np.float64, F32_TOL, F32_SIM, F32_SCORE)
 
 
 def test_random_sampling_ablation_on_ragged_batch(B):
@@ -136,7 +93,7 @@ def test_random_sampling_ablation_on_ragged_batch(B):
     p = MergeParams(merge_layers=(1, 3), tau_seg=0.6, tau_merge=0.7, selection=3, retain_mode=1, retain=0.4,
                     sample_seed=0x1234567890ABCDEF)
     wl = Workload("ragged_random", shape, "f32", vids, p, 77)
-    err, log = run_workload(B, wl, np.float64, F32_TOL, 1e-5, 1e-4)
+    err, log = run_workload(B, wl, np.float64, F32_TOL, F32_SIM, F32_SCORE)
     assert not log
 
 
@@ -159,17 +116,41 @@ def test_identical_middle_frames_collapse(B):
 
 # ------------------------------------------------------------------ bf16 tensor-core path
 
+@pytest.mark.parametrize("window_mode", [0, 1])
+def test_stage2_only_decoupled_selection(B, window_mode):
+    """No merge layer: the dynamic / static split comes from the streaming segmentation of the final features, and
+    the decoupled selection runs on it (the 'only stage 2' ablation)."""
+    shape = EncoderShape(image_size=56, patch_size=14, num_layers=4, hidden=48, heads=3, mlp_dim=100)
+    vids = (VideoSpec(9, 0.05, 3), VideoSpec(1, 0.2, 2), VideoSpec(12, 0.15, 5))
+    p = MergeParams(merge_layers=(), tau_seg=0.93, tau_merge=0.7, selection=1, retain_mode=1, retain=0.4,
+                    window_mode=window_mode)
+    wl = Workload("stage2_only", shape, "f32", vids, p, 77)
+    frames, offs = make_batch(wl)
+    res = O.encode_batch(frames, offs, shape, make_weights(shape, 77), p)
+    dyn = np.concatenate([r.frame_dynamic for r in res])
+    assert dyn.any() and not dyn.all(), "the case must have both dynamic and static frames"
+    err, log = run_workload(B, wl, np.float64, F32_TOL, F32_SIM, F32_SCORE)
+    assert not log
+
+
+def test_stage2_only_bf16(B):
+    shape = EncoderShape(image_size=70, patch_size=14, num_layers=4, hidden=144, heads=2, mlp_dim=304)
+    vids = (VideoSpec(12, 0.1, 1), VideoSpec(7, 0.3, 2))
+    p = MergeParams(merge_layers=(), tau_seg=0.5, tau_merge=0.6, selection=1, retain_mode=1, retain=0.4)
+    run_workload(B, Workload("stage2_only_bf16", shape, "bf16", vids, p, 5), np.float64, BF16_TOL, BF16_SIM, BF16_SCORE)
+
+
 def test_small_bf16_encoder(B):
     """so400m-like odd shapes at a small size: head dim 72, MLP width not a multiple of 64, ragged batch."""
     shape = EncoderShape(image_size=70, patch_size=14, num_layers=4, hidden=144, heads=2, mlp_dim=304)
     vids = (VideoSpec(12, 0.1, 1), VideoSpec(7, 0.3, 2))
     p = MergeParams(merge_layers=(1, 3), tau_seg=0.5, tau_merge=0.6, selection=1, retain_mode=1, retain=0.4)
     wl = Workload("small_bf16", shape, "bf16", vids, p, 5)
-    run_workload(B, wl, np.float64, BF16_TOL, 1e-2, 5e-2)
+    run_workload(B, wl, np.float64, BF16_TOL, BF16_SIM, BF16_SCORE)
 
 
 def test_so400m_8f_bf16(B):
-    run_workload(B, workload("so400m_8f"), np.float32, BF16_TOL, 1e-2, 5e-2)
+    run_workload(B, workload("so400m_8f"), np.float32, BF16_TOL, BF16_SIM, BF16_SCORE)
 
 
 # ------------------------------------------------------------------ host entry point and errors

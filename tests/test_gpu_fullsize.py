@@ -1,5 +1,15 @@
 """Parity at the full benchmark sizes (32, 64 and 8 x 32 frames of SigLIP-so400m shapes), in the launch
-configuration bench.py times.  The oracle cannot encode whole videos of this size in test time, so:
+configuration bench.py times.
+
+`test_full_size_against_oracle` puts the whole compressed path through the comparison protocol of tests/helpers.py
+against the oracle's results for the same seeded inputs: similarities, EMA, segments and merged pairs of every
+merge layer, attention scores, kept sets (near-ties inside the measured band logged and counted), then tokens and
+index map under identical decisions.  The numpy oracle needs 4 to 50 minutes per workload, so its results are read
+from tests/golden/fullsize_<name>.npz, written on CPU by tests/golden/make_fullsize_goldens.py (which imports only
+the oracle and the input generators); the test first checks the stored fingerprint of the oracle's inputs against
+the generators.
+
+`test_full_size_workload` adds what needs no stored values:
 
   * values: frames are independent in the uncompressed encoder, hence sampled frames of the full-size
     uncompressed run are compared with the oracle's encoding of those frames alone (<= 2e-2);
@@ -21,6 +31,9 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 BF16_TOL = 2e-2
+BF16_SIM, BF16_SCORE = 5e-4, 1e-2     # hard ceilings on similarity / score error (see tests/test_gpu_encode.py)
+NEAR_TIE_SHARE = 0.005
+FULL_SIZE = ["so400m_32f", "so400m_32f_cal", "so400m_64f_p50", "so400m_64f_p10", "so400m_64f_p90", "serve_8x32"]
 
 
 @pytest.fixture(scope="module")
@@ -100,7 +113,30 @@ def _check_structure(run, offs, L):
         np.testing.assert_array_equal(pos, np.nonzero(tr.keep[f])[0])
 
 
-@pytest.mark.parametrize("name", ["so400m_32f", "so400m_64f_p50", "so400m_64f_p10", "so400m_64f_p90", "serve_8x32"])
+@pytest.mark.parametrize("name", FULL_SIZE)
+def test_full_size_against_oracle(B, name):
+    import os
+    import torch
+    wl = workload(name)
+    assert os.path.exists(H.golden_path(name)), f"missing {H.golden_path(name)}: run tests/golden/make_fullsize_goldens.py {name}"
+    ob = H.batch_from_golden(name, len(wl.params.merge_layers))
+    frames, offs = make_batch(wl)
+    blob = make_weights(wl.shape, wl.weight_seed, wl.pos_std)
+    assert H.input_sha(frames, blob) == ob.input_sha, "the stored oracle results were computed from other inputs"
+    enc = B.Encoder(wl.shape, blob, B.ET_BF16, wl.total_frames, len(wl.videos))
+    try:
+        stats, log = H.check_parity(B, enc, torch.from_numpy(frames).cuda(), offs, wl.params, ob, BF16_TOL, BF16_SIM,
+                                    BF16_SCORE, name)
+    finally:
+        enc.close()
+    assert stats["near_ties"] <= max(1, NEAR_TIE_SHARE * stats["decisions"]), stats
+    # the budget of Eq. 5: with k near-equal windows on static frames the kept total is N*k per video
+    L = wl.shape.tokens_per_frame
+    target = wl.params.retain * wl.total_frames * L
+    assert abs(ob.n_tokens - target) <= len(ob.dynamic), (ob.n_tokens, target)
+
+
+@pytest.mark.parametrize("name", FULL_SIZE)
 def test_full_size_workload(B, name):
     import torch
     wl = workload(name)
@@ -122,6 +158,8 @@ def test_full_size_workload(B, name):
     # values: sampled frames of the uncompressed run against the oracle on those frames alone
     w = O.split_weights(shape, blob)
     samples = [0, wl.total_frames - 1] if name in ("so400m_32f", "serve_8x32") else [wl.total_frames // 2]
+    if name == "so400m_32f_cal":
+        samples = [6]                       # the first scene cut
     for fidx in samples:
         ref = O.encode_video(frames[fidx:fidx + 1], shape, w, wl.uncompressed().params, dtype=np.float32)
         err = H.token_error(unc["tokens"][fidx * L:(fidx + 1) * L], ref.tokens)
