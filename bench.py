@@ -2,6 +2,9 @@
 """Benchmark of the compressed video vision-encoder on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+    python bench.py --sweep                      timing columns of the paper's ablations, one JSON line per setting
+    python bench.py --prefill-only [--layers 28] [--vocab 152064] [--visual-tokens 7621]
+                                                 the projector + language-model prefill stage alone, per category
 
 A step is one pass of the whole hot path (patch embed, 27 blocks with Stage I at the merge layers,
 attention scores, Stage II, gather) over one synthetic 32-frame SigLIP-so400m video.  Rank 0 prints
@@ -24,8 +27,8 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of gemm_bf16_kernel<256, *> (ncu, workload so400m_32f):
-# qkv 174.7 MB, out-proj 213.4 MB, fc1 214.9 MB, fc2 401.2 MB -> average.  To be re-taken whenever that kernel changes.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of gemm_bf16_kernel<256, *>, average of the four dense
+# launches of block 0 at 32 frames (one ncu capture of this workload).  Re-taken whenever that kernel changes.
 GEMM_DRAM_BYTES_PER_LAUNCH = 251.0e6
 
 METRIC = "frames/s through compressed encoder (32f SigLIP-so400m)"
@@ -108,7 +111,8 @@ def job_throughput(ms_total_local: float, steps: int, frames_per_step_per_rank: 
 
 
 def oracle_sample(wl, frames, blob, sample_frames, steps, warmup):
-    """The CPU oracle, as it stands, on the first `sample_frames` frames of the workload's video."""
+    """The CPU oracle, as it stands, on the first `sample_frames` frames of the workload's video (the whole method:
+    Stage I can merge once a segment has four frames).  Returns (frames/s, s per step, threads, frames out, tokens out)."""
     from oracle import earlytom_oracle as O
     w = O.split_weights(wl.shape, blob)
     sub = frames[:sample_frames]
@@ -116,14 +120,21 @@ def oracle_sample(wl, frames, blob, sample_frames, steps, warmup):
         O.encode_video(sub[:1], wl.shape, w, wl.params, dtype=np.float32)
     t0 = time.perf_counter()
     for _ in range(steps):
-        O.encode_video(sub, wl.shape, w, wl.params, dtype=np.float32)
+        r = O.encode_video(sub, wl.shape, w, wl.params, dtype=np.float32)
     dt = (time.perf_counter() - t0) / steps
     try:
         from threadpoolctl import threadpool_info
         cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
         cores = os.cpu_count() or 1
-    return sample_frames / dt, dt, cores
+    return sample_frames / dt, dt, cores, len(r.frame_dynamic), int(r.tokens.shape[0])
+
+
+def sample_note(sample, total, frames_out, tokens_out, L):
+    merged = "no merge executed: Stage I needs four frames in a segment" if sample < 4 else \
+        f"Stage I left {frames_out} of {sample} frames"
+    return (f"first {sample} of {total} frames of the same video, numpy fp32 oracle, whole method ({merged}; "
+            f"{tokens_out} of {sample * L} tokens kept)")
 
 
 def run_reference(args, wl):
@@ -133,15 +144,17 @@ def run_reference(args, wl):
         return
     frames, _ = make_batch(wl)
     blob = make_weights(wl.shape, wl.weight_seed, wl.pos_std)
-    # one frame per step keeps the default --steps 20 run within a few minutes on the machine's host cores
-    sample = 1
-    fps, dt, cores = oracle_sample(wl, frames, blob, sample, max(1, args.steps), min(1, args.warmup))
+    # The oracle needs 6-10 s per frame on 8-16 host cores.  The sample per step is sized so that the whole
+    # --steps K run stays near three minutes: 8 frames per step (Stage I merges) up to K = 3, one frame at K = 20.
+    steps = max(1, args.steps)
+    sample = int(max(1, min(8, wl.videos[0].n_frames, 24 // steps)))
+    fps, dt, cores, n_out, t_out = oracle_sample(wl, frames, blob, sample, steps, min(1, args.warmup))
+    note = sample_note(sample, wl.total_frames, n_out, t_out, wl.shape.tokens_per_frame)
     line = {"impl": "reference", "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "frames": wl.total_frames, "sample": f"first {sample} frame(s) of the video per step"},
-            "cpu_baseline": {"value": fps, "unit": UNIT, "cores": cores, "kind": "oracle",
-                             "sample": f"first {sample} of {wl.total_frames} frames of the same video, numpy fp32 oracle"},
+            "config": {"workload": wl.name, "frames": wl.total_frames, "sample": note},
+            "cpu_baseline": {"value": fps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": note},
             "e2e": {"value": fps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -166,14 +179,24 @@ def run_sweep(args, wl, enc, dev_vids, offs, n_rot, stream, barrier, torch):
                  ("stage II only", replace(base, merge_layers=()))]
     steps = max(3, args.steps // 4)
     ref_ms = None
+    from synthetic import make_video, workload
+    cal = workload("so400m_32f_cal")
+    if wl.name == "so400m_32f":        # the same setting on the video with scene cuts (Stage I keeps about 3/4 of the frames)
+        cv = cal.videos[0]
+        cal_vids = [torch.from_numpy(make_video(cv.n_frames, wl.shape.image_size, wl.shape.patch_size, cv.resample_p,
+                                                cv.seed + sd, cv.jitter, cv.cut_every)).cuda() for sd in range(n_rot)]
+        settings.append(("main setting, video with a scene cut every 6 frames", None))
     for name, p in settings:
+        vids_here = dev_vids
+        if p is None:
+            p, vids_here = base, cal_vids
         for i in range(2):
-            res = enc.encode_batch(dev_vids[i % n_rot], offs, p)
+            res = enc.encode_batch(vids_here[i % n_rot], offs, p)
         barrier()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record(stream)
         for i in range(steps):
-            res = enc.encode_batch(dev_vids[i % n_rot], offs, p)
+            res = enc.encode_batch(vids_here[i % n_rot], offs, p)
         ev1.record(stream)
         barrier()
         ms = ev0.elapsed_time(ev1) / steps
@@ -248,6 +271,117 @@ def run_downstream(args, wl, enc, dev_vids, offs, stream, peaks, torch, B):
                                      "launches": sum(prof_main["launches"].values()) // calls}}
 
 
+def run_parity(wl, B, torch):
+    """The comparison protocol of the GPU tests on this workload's seeded input against the oracle's stored results
+    (tests/golden/fullsize_<name>.npz, written on CPU by tests/golden/make_fullsize_goldens.py): similarities,
+    decisions, scores, kept sets with the near-tie log, tokens under identical decisions.  Returns the summary."""
+    from synthetic import make_batch, make_weights
+    from tests import helpers as H
+    if not os.path.exists(H.golden_path(wl.name)):
+        return {"config": wl.name, "skipped": "no stored oracle results for this workload"}
+    ob = H.batch_from_golden(wl.name, len(wl.params.merge_layers))
+    frames, offs = make_batch(wl)
+    blob = make_weights(wl.shape, wl.weight_seed, wl.pos_std)
+    if H.input_sha(frames, blob) != ob.input_sha:
+        return {"config": wl.name, "skipped": "stored oracle results belong to other inputs"}
+    enc = B.Encoder(wl.shape, blob, B.ET_BF16 if wl.dtype == "bf16" else B.ET_F32, wl.total_frames, len(wl.videos))
+    try:
+        import contextlib
+        import io
+        with contextlib.redirect_stdout(io.StringIO()):
+            stats, log = H.check_parity(B, enc, torch.from_numpy(frames).cuda(), list(offs), wl.params, ob, 2e-2, 5e-4, 1e-2, wl.name)
+        stats["passed"] = True
+        stats["near_tie_log"] = log[:16]
+    except AssertionError as ex:
+        stats = {"config": wl.name, "passed": False, "error": str(ex)[:300]}
+    finally:
+        enc.close()
+    return stats
+
+
+def run_hbm_kernels(args, B, torch, peaks, name="serve_8x32"):
+    """The bandwidth-bound kernels on a workload whose residual stream (430 MB of fp32 at 8 x 32 frames) does not
+    fit the 126 MB L2, so that their GB/s are DRAM figures: a few profiled steps of the whole path, per category."""
+    from synthetic import make_batch, make_weights, workload
+    wl = workload(name)
+    frames, offs = make_batch(wl)
+    blob = make_weights(wl.shape, wl.weight_seed, wl.pos_std)
+    enc = B.Encoder(wl.shape, blob, B.ET_BF16, wl.total_frames, len(wl.videos))
+    try:
+        fr = torch.from_numpy(frames).cuda()
+        for _ in range(2):
+            res = enc.encode_batch(fr, list(offs), wl.params)
+        B.et_profile_enable(enc, True)
+        steps = 3
+        for _ in range(steps):
+            res = enc.encode_batch(fr, list(offs), wl.params)
+        torch.cuda.synchronize()
+        prof = B.et_profile_read(enc)
+        B.et_profile_enable(enc, False)
+        out = {"workload": name, "frames": wl.total_frames, "frames_out": res.n_frames_out, "tokens_out": res.n_tokens,
+               "steps": steps, "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"] + " (copy bandwidth)"}
+        for cat in ("similarity", "merge", "gather", "layernorm", "select", "im2col"):
+            c = prof[cat]
+            if c["ms"] <= 0:
+                continue
+            gbs = c["work"] / (c["ms"] * 1e-3) / 1e9
+            out[cat] = {"gbs": round(gbs, 1), "frac": round(gbs / peaks["hbm_gbs"], 3), "bytes_per_step": c["work"] / prof["calls"],
+                        "ms_per_step": round(c["ms"] / prof["calls"], 4), "launches_per_step": c["launches"] / prof["calls"]}
+        g = prof["gemm"]
+        out["gemm_tflops"] = round(g["work"] / (g["ms"] * 1e-3) / 1e12, 1)
+        out["ms_per_step"] = round(sum(prof[c]["ms"] for c in B.PROF_NAMES) / prof["calls"], 3)
+        return out
+    finally:
+        enc.close()
+
+
+def run_prefill_only(args):
+    """The projector + language-model prefill stage alone, per kernel category, on random-init weights drawn on the
+    device (Qwen2-7B widths by default; --layers / --vocab shrink the model so that a profiler capture stays small)."""
+    from dataclasses import replace
+    import torch
+    from paper_2605_30010_b200 import binding as B
+    from synthetic.llm import QWEN2_7B, make_llm_weights_device, make_prompt, make_visual_tokens
+    shape = replace(QWEN2_7B, num_layers=args.layers, vocab=args.vocab)
+    blob = make_llm_weights_device(shape, 5)
+    llm = B.LanguageModel(shape, blob, max_tokens=args.visual_tokens + 64, keep_kv_cache=True)
+    del blob
+    torch.cuda.empty_cache()
+    pre, suf = make_prompt(shape, 14, 40, 6)
+    vis = torch.from_numpy(make_visual_tokens(shape, args.visual_tokens, 6)).cuda()
+    iters = max(1, args.steps)
+    for _ in range(max(1, args.warmup)):
+        B.et_llm_prefill(llm, pre, vis, suf, copy_logits=False)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        r = B.et_llm_prefill(llm, pre, vis, suf, copy_logits=False)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    B.et_llm_profile_enable(llm, True)
+    for _ in range(iters):
+        B.et_llm_prefill(llm, pre, vis, suf, copy_logits=False)
+    p = B.et_llm_profile_read(llm)
+    llm.close()
+    n, calls = r.n_tokens, p["calls"]
+    H, M, L = shape.hidden, shape.mlp_dim, shape.num_layers
+    per = {k: v / calls for k, v in p["ms"].items()}
+    gemm_flops = L * 2.0 * n * (H * shape.qkv_dim + shape.q_dim * H + 3 * H * M) \
+        + 2.0 * args.visual_tokens * (shape.vision_hidden * H + H * H) + 2.0 * H * shape.vocab
+    attn_flops = L * 2.0 * n * n * shape.q_dim                # causal: half of the n^2 products
+    norm_bytes = 2 * L * n * H * (4 + 2)                      # fp32 row in, bf16 row out
+    rope_bytes = L * n * (shape.q_dim + shape.kv_dim) * 2 * 2   # Q and K parts read and written
+    print(json.dumps({"tokens": n, "layers": L, "vocab": shape.vocab, "ms_per_prefill": round(ms, 3),
+                      "tokens_per_s": round(n / (ms * 1e-3), 1), "ms_per_category": {k: round(v, 4) for k, v in per.items()},
+                      "launches_per_prefill": {k: v // calls for k, v in p["launches"].items()},
+                      "gemm_tflops": round(gemm_flops / (per["gemm"] * 1e-3) / 1e12, 1),
+                      "attention_tflops": round(attn_flops / (per["attention"] * 1e-3) / 1e12, 1),
+                      "rmsnorm_gbs": round(norm_bytes / (per["norm"] * 1e-3) / 1e9, 1),
+                      "rope_gbs": round(rope_bytes / (per["rope"] * 1e-3) / 1e9, 1)}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -261,7 +395,16 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark line, time the paper's ablation settings (merge start layer, retained "
                          "ratio, sampling strategy, single stages) on the workload and print one JSON line per setting")
+    ap.add_argument("--no-parity", action="store_true", help="skip the parity summary against the stored oracle results")
+    ap.add_argument("--no-hbm-kernels", action="store_true",
+                    help="skip the profiled steps of the 8 x 32-frame workload (DRAM figures of the bandwidth kernels)")
+    ap.add_argument("--prefill-only", action="store_true", help="time the projector + language-model prefill stage alone")
+    ap.add_argument("--layers", type=int, default=28, help="--prefill-only: decoder layers")
+    ap.add_argument("--vocab", type=int, default=152064, help="--prefill-only: vocabulary size")
+    ap.add_argument("--visual-tokens", type=int, default=7621, help="--prefill-only: visual tokens in the sequence")
     args = ap.parse_args()
+    if args.prefill_only:
+        return run_prefill_only(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from synthetic import make_video, make_weights, workload
@@ -386,7 +529,7 @@ def main():
                 "launches": g["launches"], "avg_launch_ms": g["ms"] / max(1, g["launches"]),
                 "traffic": GEMM_DRAM_BYTES_PER_LAUNCH if wl.name == "so400m_32f" else None,
                 "traffic_unit": "bytes per launch (dram read + written), average of the four dense launches of block 0 at "
-                                "32 frames, from the ncu capture summarised in profiles/gemm_bf16_kernel_so400m_32f.md"}
+                                "32 frames, one ncu capture"}
     per_cat = {}
     for name in B.PROF_NAMES:
         c = prof[name]
@@ -406,8 +549,11 @@ def main():
             "dtype": wl.dtype, "data": "synthetic",
             "config": {"workload": wl.name, "videos": V, "frames": T, "tokens_per_frame": shape.tokens_per_frame,
                        "merge_layers": list(params.merge_layers), "tau_seg": params.tau_seg, "tau_merge": params.tau_merge,
-                       "retain": params.retain, "frames_per_block": res.frames_per_block, "frames_out": res.n_frames_out,
-                       "tokens_out": res.n_tokens, "parallelism": f"replicas x{world}",
+                       "retain": params.retain, "window_mode": params.window_mode,
+                       "frames_per_block": res.frames_per_block, "frames_out": res.n_frames_out,
+                       "stage1_frames_out": res.n_frames_out, "stage1_frame_retention": round(res.n_frames_out / T, 4),
+                       "tokens_out": res.n_tokens, "retained_ratio": round(res.n_tokens / (T * shape.tokens_per_frame), 4),
+                       "parallelism": f"replicas x{world}",
                        "l2": f"inputs rotate over {n_rot} videos; weights (824 MB) + activations per step exceed the 126 MB L2"},
             "ms_per_video": ms_step, "clocks": clocks, "gpu_launches": int(launches),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -419,11 +565,22 @@ def main():
             line["downstream"] = run_downstream(args, wl, enc, dev_vids, offs, stream, peaks, torch, B)
         except Exception as ex:          # the headline line never depends on this stage
             line["downstream"] = {"error": f"{type(ex).__name__}: {ex}"}
+    enc.close()
+    if not args.no_parity and world == 1:
+        try:
+            line["parity"] = run_parity(wl, B, torch)
+        except Exception as ex:
+            line["parity"] = {"config": wl.name, "passed": False, "error": f"{type(ex).__name__}: {ex}"[:300]}
+    if not args.no_hbm_kernels and world == 1 and wl.name == "so400m_32f":
+        try:
+            line["hbm_kernels"] = run_hbm_kernels(args, B, torch, peaks)
+        except Exception as ex:
+            line["hbm_kernels"] = {"error": f"{type(ex).__name__}: {ex}"[:300]}
     if not args.no_cpu_baseline:
-        sample = 2
-        fps, dt, cores = oracle_sample(wl, vids[0], blob, sample, 1, 1)
+        sample = min(8, wl.videos[0].n_frames)
+        fps, dt, cores, n_out, t_out = oracle_sample(wl, vids[0], blob, sample, 1, 1)
         line["cpu_baseline"] = {"value": fps, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"first {sample} of {T} frames of one video, numpy fp32 oracle, {dt:.1f} s"}
+                                "sample": sample_note(sample, T, n_out, t_out, shape.tokens_per_frame) + f", {dt:.1f} s"}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -192,8 +192,8 @@ enum {
   ET_CAT_GEMM = 1,      /* flops: 2*M*N*K of every dense layer (patch embed, QKV, out-proj, MLP) */
   ET_CAT_ATTENTION = 2, /* flops: 4*L*L*D per frame per block */
   ET_CAT_LAYERNORM = 3, /* bytes: rows*D*(4 + output element size) */
-  ET_CAT_SIMILARITY = 4,/* bytes: n*L*D*4 read once + cosines written and re-read */
-  ET_CAT_PLAN = 5,      /* bytes: 0 (latency-bound scalar work) */
+  ET_CAT_SIMILARITY = 4,/* bytes: n*L*D*4 read once (includes the merge plan, same launch) */
+  ET_CAT_PLAN = 5,      /* unused: the plan runs in the tail of the similarity launch */
   ET_CAT_MERGE = 6,     /* bytes: source frames read + output frames written */
   ET_CAT_SCORES = 7,    /* flops: 2*L*L*D per output frame */
   ET_CAT_SELECT = 8,    /* bytes: scores read + mask written */
@@ -209,6 +209,21 @@ typedef struct {
 /* on != 0: reset the counters and start collecting; 0: stop. */
 ET_API et_status et_profile_enable(et_encoder* enc, int on);
 ET_API et_status et_profile_read(const et_encoder* enc, et_profile* out);
+
+/* Self-test of the failure-detection path (no counterpart in the paper).  Every tensor-core kernel of the library
+ * waits on its barriers with a time limit and, when the limit runs out, records a status word, releases what it
+ * holds and returns, which the encode calls report as ET_ERR_TIMEOUT.  This call runs that same bounded wait in a
+ * one-warp kernel on a barrier that expects one arrival: with arrive = 0 nothing arrives, the wait runs out after
+ * limit_ns (1 .. 1e9 nanoseconds) and the call returns ET_ERR_TIMEOUT; with arrive = 1 a lane arrives and the call
+ * returns ET_OK.  Synchronous; the context stays usable either way. */
+ET_API et_status et_selftest_bounded_wait(unsigned long long limit_ns, int arrive, void* cuda_stream);
+
+/* The checked build (libearlytom_debug.so, compiled with -DET_DEBUG) verifies the indices the Stage I, Stage II and
+ * gather kernels compute before using them; a bad index is recorded and the access skipped (nothing traps).
+ * et_debug_build() says whether this library is that build; et_debug_status() returns 0 if no check has failed
+ * since the library was loaded (always 0 in the regular build), non-zero otherwise. */
+ET_API int et_debug_build(void);
+ET_API int et_debug_status(void);
 
 /* Number of kernels the library has launched in this process (all encoders); for benchmarks. */
 ET_API unsigned long long et_kernel_launch_count(void);
@@ -236,7 +251,8 @@ ET_API et_status et_frame_similarity(const float* x_dev, int n, int L, int D, fl
  *   - the call itself never allocates or frees; every GPU that loads the library holds the array
  *     until the process exits;
  *   - the first call on each device looks up the array's device address (host-side, once); make
- *     that first call before any stream capture begins;
+ *     that first call before any stream capture begins; the address is remembered per device, so a
+ *     process that calls cudaDeviceReset must not use this entry point on that device afterwards;
  *   - the array is shared by all calls and keeps the last call's cosines; nothing needs clearing
  *     (every value read is written first), but calls that overlap on the GPU race on it. */
 ET_API et_status et_frame_similarity_static(const float* x_dev, int n, int L, int D, float* sim_dev,

@@ -13,7 +13,8 @@ from typing import List, Optional, Sequence
 
 import numpy as np
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libearlytom.so")
+# EARLYTOM_LIB selects another build of the same library (the checked build libearlytom_debug.so)
+_LIB_PATH = os.environ.get("EARLYTOM_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libearlytom.so")
 
 ET_F32, ET_BF16 = 0, 1
 ET_MAX_MERGE_LAYERS = 8
@@ -21,6 +22,7 @@ STATUS_NAMES = ["ET_OK", "ET_ERR_INVALID_ARG", "ET_ERR_SHAPE", "ET_ERR_CAPACITY"
                 "ET_ERR_TIMEOUT", "ET_ERR_WEIGHTS"]
 EXPORTS = ["et_encoder_create", "et_encode_video", "et_encode_batch", "et_encode_batch_host", "et_destroy",
            "et_status_string", "et_last_error", "et_kernel_launch_count", "et_profile_enable", "et_profile_read",
+           "et_selftest_bounded_wait", "et_debug_build", "et_debug_status",
            "et_frame_similarity_static", "et_frame_similarity", "et_merge_plan",
            "et_merge_frames", "et_select_tokens", "et_gather_tokens", "et_linear_bf16", "et_attention",
            "et_attention_scores", "et_layernorm",
@@ -140,6 +142,9 @@ def load_library(path: str = _LIB_PATH) -> C.CDLL:
     lib.et_last_error.restype = C.c_char_p
     lib.et_kernel_launch_count.argtypes = []
     lib.et_kernel_launch_count.restype = C.c_ulonglong
+    lib.et_selftest_bounded_wait.argtypes = [C.c_ulonglong, i, vp]
+    lib.et_debug_build.argtypes = []
+    lib.et_debug_status.argtypes = []
     lib.et_profile_enable.argtypes = [vp, i]
     lib.et_profile_read.argtypes = [vp, C.POINTER(et_profile)]
     lib.et_frame_similarity.argtypes = [vp, i, i, i, vp, vp, vp]
@@ -429,6 +434,19 @@ def et_encode_batch_host(enc: Encoder, frames_host, video_offsets: Sequence[int]
 
 def et_kernel_launch_count() -> int:
     return int(lib().et_kernel_launch_count())
+
+
+def et_selftest_bounded_wait(limit_ns: int, arrive: bool, stream=None) -> None:
+    """Raises EarlyTomError(ET_ERR_TIMEOUT) when the wait runs out (arrive = False)."""
+    _check(lib().et_selftest_bounded_wait(C.c_ulonglong(int(limit_ns)), 1 if arrive else 0, _stream_ptr(stream)))
+
+
+def et_debug_build() -> bool:
+    return bool(lib().et_debug_build())
+
+
+def et_debug_status() -> int:
+    return int(lib().et_debug_status())
 
 
 def et_profile_enable(enc: Encoder, on: bool) -> None:

@@ -1,9 +1,11 @@
 """Builds libearlytom.so (all CUDA sources of csrc/) for sm_100a with nvcc, in-tree.
 
-    python -m paper_2605_30010_b200.build [--force] [--verbose]
+    python -m paper_2605_30010_b200.build [--force] [--verbose] [--debug]
 
 Objects go to <repo>/_build (ignored by git); the shared library lands in
 paper_2605_30010_b200/lib/libearlytom.so.  nvcc cross-compiles without a GPU.
+--debug builds the checked variant (-DET_DEBUG: index checks in the Stage I / Stage II / gather
+kernels that record a status instead of faulting) as lib/libearlytom_debug.so from _build/debug.
 """
 from __future__ import annotations
 
@@ -16,6 +18,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "lib", "libearlytom.so")
+LIB_DEBUG = os.path.join(PKG, "lib", "libearlytom_debug.so")
 OBJ_DIR = os.path.join(ROOT, "_build")
 
 NVCC_FLAGS = [
@@ -36,18 +39,21 @@ def _deps_mtime():
     return max(os.path.getmtime(f) for f in files)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    os.makedirs(OBJ_DIR, exist_ok=True)
-    os.makedirs(os.path.dirname(LIB), exist_ok=True)
+    obj_dir = os.path.join(OBJ_DIR, "debug") if debug else OBJ_DIR
+    lib_path = LIB_DEBUG if debug else LIB
+    flags = NVCC_FLAGS + (["-DET_DEBUG"] if debug else [])
+    os.makedirs(obj_dir, exist_ok=True)
+    os.makedirs(os.path.dirname(lib_path), exist_ok=True)
     hdr = _deps_mtime()
     jobs = []
     objs = []
     for src in sources():
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr):
-            cmd = [nvcc, *NVCC_FLAGS, "-c", src, "-o", obj]
+            cmd = [nvcc, *flags, "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas")
                 cmd.insert(2, "-v")
@@ -65,15 +71,15 @@ def build(force: bool = False, verbose: bool = False) -> str:
             failed |= r.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    if jobs or force or not os.path.exists(LIB):
-        cmd = [nvcc, "-shared", "-o", LIB, *objs, "-gencode", "arch=compute_100a,code=sm_100a",
+    if jobs or force or not os.path.exists(lib_path):
+        cmd = [nvcc, "-shared", "-o", lib_path, *objs, "-gencode", "arch=compute_100a,code=sm_100a",
                "-Xcompiler", "-fPIC"]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)
             raise RuntimeError("link failed")
-    return LIB
+    return lib_path
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

@@ -21,8 +21,33 @@ enum DeviceStatus : int {
   DS_OK = 0,
   DS_WAIT_EXPIRED = 1,      // a bounded mbarrier wait ran out
   DS_FORCED_MISMATCH = 2,   // forced plan does not fit the frame list on the device
-  DS_CAPACITY = 3
+  DS_CAPACITY = 3,
+  DS_BAD_INDEX = 4          // checked build only: an index left its array
 };
+
+// Index checks of the checked build (-DET_DEBUG, libearlytom_debug.so): a violated condition records DS_BAD_INDEX in
+// a status word of the translation unit (read by et_debug_status) and the statement `skip` is executed instead
+// of the access; nothing traps.  In the regular build the macro expands to nothing.
+#ifdef ET_DEBUG
+#define ET_DEBUG_STATUS_WORD static __device__ int g_debug_status_word = 0;
+#define ET_CHECK(cond, skip)                                  \
+  do {                                                        \
+    if (!(cond)) {                                            \
+      atomicExch(&g_debug_status_word, (int)::et::DS_BAD_INDEX); \
+      skip;                                                   \
+    }                                                         \
+  } while (0)
+#define ET_DEBUG_STATUS_READ(fn)                                                        \
+  int fn() {                                                                            \
+    int v = 0;                                                                          \
+    if (cudaMemcpyFromSymbol(&v, g_debug_status_word, sizeof(int)) != cudaSuccess) return -1; \
+    return v;                                                                           \
+  }
+#else
+#define ET_DEBUG_STATUS_WORD
+#define ET_CHECK(cond, skip) do { } while (0)
+#define ET_DEBUG_STATUS_READ(fn) int fn() { return 0; }
+#endif
 
 static inline int cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
 
@@ -157,27 +182,46 @@ struct PlanArgs {
   int* n_hist_slot;              // receives the new frame count (may be NULL)
   int* status;
 };
-void launch_merge_plan(const PlanArgs& a, cudaStream_t s);
+void launch_merge_plan(const PlanArgs& a, int n_cap, cudaStream_t s);
+// Similarities of the current list and its plan in one launch (no scratch array, no kernel waits: see stage1.cu).
+// acc: similarity_plan_words(n_cap) - 1 64-bit accumulators and done: [1] ticket counter, zero before the first
+// launch; every launch leaves them at zero.
+struct SimPlanArgs {
+  const float* x;               // [n_cap][L][D] residual stream
+  float* sim;                   // [n_cap]; must be plan.sim
+  int n_cap, L, D;
+  const int* n_frames_dev;      // live frames
+  const int* vid_off;           // [n_videos+1] of the current list
+  int n_videos;
+  unsigned long long* acc;      // [slots][n_cap]
+  unsigned* done;               // [1]
+  PlanArgs plan;
+};
+void launch_similarity_plan(const SimPlanArgs& a, cudaStream_t s);
+int similarity_plan_words(int n_cap);
 void launch_merge_frames(const float* x, float* y, int n_cap, int frame_elems, const int* n_out_dev,
                          const MergePlan& plan, cudaStream_t s);
 void launch_init_frames(const FrameList& fl, const int* vid_off_src_dev, int n_videos, int n_frames, cudaStream_t s);
 
 // ---- stage2.cu -----------------------------------------------------------------------------
-struct SelectSetupArgs {
-  FrameList fl;
+struct SelectArgs {
+  const float* scores;       // [n_cap][L]
+  FrameList fl;              // current list: live count, video offsets, roles
   const int* orig_vid_off;   // [V+1] offsets of the input videos (for B of Eq. 5)
-  int n_videos, L, selection, retain_mode;
+  int n_cap, n_videos, L, selection, retain_mode, window_mode;
+  int mask_given;            // 1: keep[] was provided by the caller; write only the flags and amounts
   double retain;
   unsigned char* dynamic;    // [Fmax] out
-  int* k_frame;              // [Fmax] out
-  int* w_frame;              // [Fmax] out
+  unsigned char* keep;       // [Fmax][L] out
+  int* count;                // [Fmax] out
   int* video_k;              // [Vmax] out
   int* video_w;              // [Vmax] out
 };
-void launch_select_setup(const SelectSetupArgs& a, int n_cap, cudaStream_t s);
+// per-video amounts (Eq. 5-6), per-frame dynamic flags and the keep mask in one launch
+void launch_select_video_tokens(const SelectArgs& a, cudaStream_t s);
+// keep mask from per-frame amounts given by the caller (the single-step entry point)
 void launch_select_tokens(const float* scores, const unsigned char* dynamic, const int* k_frame, const int* w_frame,
-                          int n_cap, int L, int selection_all, int window_mode, unsigned char* keep, int* count,
-                          const int* n_frames_dev, cudaStream_t s);
+                          int n_cap, int L, int window_mode, unsigned char* keep, int* count, cudaStream_t s);
 // Random-sampling ablation: scores[f][j] = uniform number of Philox-4x32-10 with counter (j, frame inside its
 // video, video, 0) and key = seed, for the frames of the current list.
 void launch_random_scores(float* scores, const int* vid_off, int n_videos, int n_cap, int L, unsigned long long seed,
@@ -186,8 +230,10 @@ void launch_count_keep(const unsigned char* keep, int n_cap, int L, int* count, 
 // frame_offsets[0..n] = exclusive scan of count; totals[0] = n_frames, totals[1] = n_tokens
 void launch_scan_counts(const int* count, int* frame_offsets, int* totals, int n_cap, const int* n_frames_dev,
                         cudaStream_t s);
-void launch_gather_tokens(const float* x, const unsigned char* keep, const int* frame_offsets, int n_cap, int L, int D,
-                          const float* ln_g, const float* ln_b, float eps, float* tokens, int* token_pos,
-                          const int* n_frames_dev, cudaStream_t s);
+// gathers the kept rows; also writes frame_offsets[0..n] (exclusive scan of count) and totals[0] = n_frames,
+// totals[1] = n_tokens
+void launch_gather_tokens(const float* x, const unsigned char* keep, const int* count, int* frame_offsets, int* totals,
+                          int n_cap, int L, int D, const float* ln_g, const float* ln_b, float eps, float* tokens,
+                          int* token_pos, const int* n_frames_dev, cudaStream_t s);
 
 }  // namespace et

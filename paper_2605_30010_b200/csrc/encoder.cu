@@ -34,6 +34,14 @@ __global__ void transpose_to_bf16_kernel(const float* __restrict__ src, bf16* __
   }
 }
 
+// flag[0] = 1 if any of the `count` floats is NaN or infinite
+__global__ void find_nonfinite_kernel(const float* __restrict__ w, size_t count, int* __restrict__ flag) {
+  bool bad = false;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x)
+    bad |= !isfinite(w[i]);
+  if (__syncthreads_or(bad) && threadIdx.x == 0) atomicExch(flag, 1);
+}
+
 struct LayerOffsets { size_t ln1_g, ln1_b, wqkv, bqkv, wo, bo, ln2_g, ln2_b, w1, b1, w2, b2; };
 
 struct LayerBf16 {
@@ -69,7 +77,7 @@ struct et_encoder {
   TmaDesc c_X[2], c_QKV, c_Hm;                      // output (C) maps
   AttnMaps attn_maps;                               // QKV as seen by the tcgen05 attention kernel
   bool attn_tc = false;
-  float *lse = nullptr, *score_partial = nullptr, *scores = nullptr, *cosbuf = nullptr, *simbuf = nullptr;
+  float *lse = nullptr, *score_partial = nullptr, *scores = nullptr, *simbuf = nullptr;
   float* frames_stage = nullptr;               // device staging for the *_host entry point (lazy)
 
   // frame lists, plans, traces
@@ -80,7 +88,8 @@ struct et_encoder {
   unsigned char* forced_mrg[ET_MAX_MERGE_LAYERS]{};
   int* orig_vid_off = nullptr;
   unsigned char *dynamic = nullptr, *keep = nullptr;
-  int *k_frame = nullptr, *w_frame = nullptr, *video_k = nullptr, *video_w = nullptr, *count = nullptr;
+  int *video_k = nullptr, *video_w = nullptr, *count = nullptr;
+  unsigned long long* sim_acc = nullptr;        // [Fmax] similarity accumulators + the ticket word (zero between launches)
   int *frame_offsets = nullptr, *token_pos = nullptr;
   float* tokens = nullptr;
   int* d_small = nullptr;   // [0] n_frames, [1] n_tokens, [2..9] n after merge layer i, [10] status
@@ -225,6 +234,15 @@ et_status dense(et_encoder* e, const void* a, const TmaDesc& da, const float* w_
   return ET_OK;
 }
 
+SimPlanArgs sim_plan_args(et_encoder* e, const float* x, int n_cap, int lst, int V, const PlanArgs& plan) {
+  SimPlanArgs a{};
+  a.x = x; a.sim = e->simbuf; a.n_cap = n_cap; a.L = e->L; a.D = e->cfg.hidden;
+  a.n_frames_dev = e->fl[lst].n; a.vid_off = e->fl[lst].vid_off; a.n_videos = V;
+  a.acc = e->sim_acc; a.done = reinterpret_cast<unsigned*>(e->sim_acc + (similarity_plan_words(e->Fmax) - 1));
+  a.plan = plan;
+  return a;
+}
+
 et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off_host, int V, const et_params* p,
                       cudaStream_t s, et_result* out) {
   if (!e || !frames_dev || !vid_off_host || !out) return fail(e, ET_ERR_INVALID_ARG, "null argument");
@@ -279,10 +297,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
   int mi = 0;
   for (int layer = 0; layer < c.num_layers; ++layer) {
     if (mi < p->num_merge_layers && p->merge_layers[mi] == layer) {
-      // Stage I at this block: similarities -> plan -> weighted merge + compaction
-      const int* n_dev = e->fl[lst].n;
-      PROF(ET_CAT_SIMILARITY, launch_token_cosines(e->X[cur], e->cosbuf, T, L, D, n_dev, s));
-      PROF(ET_CAT_SIMILARITY, launch_reduce_cosines(e->cosbuf, e->simbuf, T, L, n_dev, s));
+      // Stage I at this block: similarities + plan (one launch) -> weighted merge + compaction
       PlanArgs a{};
       a.sim = e->simbuf; a.cur = e->fl[lst]; a.nxt = e->fl[lst ^ 1]; a.plan = e->plan; a.trace = e->tr[mi];
       a.forced_seg_start = fp ? e->forced_seg[mi] : nullptr;
@@ -291,7 +306,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
       a.alpha = p->ema_alpha; a.tau_seg = p->tau_seg; a.tau_merge = p->tau_merge;
       a.weighted = p->weighted_merge; a.allow_merge = 1; a.n_videos = V;
       a.n_hist_slot = e->d_small + 2 + mi; a.status = e->d_small + 10;
-      PROF(ET_CAT_PLAN, launch_merge_plan(a, s));
+      PROF(ET_CAT_SIMILARITY, launch_similarity_plan(sim_plan_args(e, e->X[cur], T, lst, V, a), s));
       PROF(ET_CAT_MERGE, launch_merge_frames(e->X[cur], e->X[cur ^ 1], T, L * D, e->fl[lst ^ 1].n, e->plan, s));
       cur ^= 1; lst ^= 1; ++mi;
     }
@@ -325,38 +340,33 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
   const int* n_dev = e->fl[lst].n;
   if (p->num_merge_layers == 0) {
     // Stage I off: the segment list of Stage II comes from the streaming segmentation of the final features
-    PROF(ET_CAT_SIMILARITY, launch_token_cosines(e->X[cur], e->cosbuf, T, L, D, n_dev, s));
-    PROF(ET_CAT_SIMILARITY, launch_reduce_cosines(e->cosbuf, e->simbuf, T, L, n_dev, s));
     PlanArgs a{};
     a.sim = e->simbuf; a.cur = e->fl[lst]; a.nxt = e->fl[lst ^ 1]; a.plan = e->plan; a.trace = e->tr[0];
     a.alpha = p->ema_alpha; a.tau_seg = p->tau_seg; a.tau_merge = p->tau_merge;
     a.weighted = p->weighted_merge; a.allow_merge = 0; a.n_videos = V; a.status = e->d_small + 10;
-    PROF(ET_CAT_PLAN, launch_merge_plan(a, s));
+    PROF(ET_CAT_SIMILARITY, launch_similarity_plan(sim_plan_args(e, e->X[cur], T, lst, V, a), s));
   }
-  // Stage II
-  SelectSetupArgs sa{};
-  sa.fl = e->fl[lst]; sa.orig_vid_off = e->orig_vid_off; sa.n_videos = V; sa.L = L; sa.selection = p->selection;
-  sa.retain_mode = p->retain_mode; sa.retain = p->retain; sa.dynamic = e->dynamic; sa.k_frame = e->k_frame;
-  sa.w_frame = e->w_frame; sa.video_k = e->video_k; sa.video_w = e->video_w;
-  PROF(ET_CAT_SELECT, launch_select_setup(sa, T, s));
+  // Stage II: amounts, flags and mask in one launch; offsets, totals and the gather in another
+  SelectArgs sa{};
+  sa.scores = e->scores; sa.fl = e->fl[lst]; sa.orig_vid_off = e->orig_vid_off; sa.n_cap = T; sa.n_videos = V; sa.L = L;
+  sa.selection = p->selection; sa.retain_mode = p->retain_mode; sa.window_mode = p->window_mode; sa.retain = p->retain;
+  sa.dynamic = e->dynamic; sa.keep = e->keep; sa.count = e->count; sa.video_k = e->video_k; sa.video_w = e->video_w;
   if (fp && fp->keep) {
     memcpy(e->h_keep_stage, fp->keep, (size_t)fp->n_final * L);
     ET_CUDA(e, cudaMemcpyAsync(e->keep, e->h_keep_stage, (size_t)fp->n_final * L, cudaMemcpyHostToDevice, s));
+    sa.mask_given = 1;
+    PROF(ET_CAT_SELECT, launch_select_video_tokens(sa, s));
     PROF(ET_CAT_SELECT, launch_count_keep(e->keep, T, L, e->count, n_dev, s));
   } else {
-    const bool rank_all = p->selection == 2 || p->selection == 3;
-    const float* sel_scores = e->scores;
     if (p->selection == 3) {          // random sampling: rank uniform numbers instead of attention scores
       PROF(ET_CAT_SELECT, launch_random_scores(e->score_partial, e->fl[lst].vid_off, V, T, L, p->sample_seed, n_dev, s));
-      sel_scores = e->score_partial;
+      sa.scores = e->score_partial;
     }
-    if (rank_all) ET_CUDA(e, cudaMemsetAsync(e->dynamic, 1, T, s));            // every frame ranks globally
-    PROF(ET_CAT_SELECT, launch_select_tokens(sel_scores, e->dynamic, e->k_frame, e->w_frame, T, L, p->selection == 0, p->window_mode, e->keep, e->count, n_dev, s));
-    if (rank_all) PROF(ET_CAT_SELECT, launch_select_setup(sa, T, s));          // restore the reported dynamic flags
+    PROF(ET_CAT_SELECT, launch_select_video_tokens(sa, s));
   }
-  PROF(ET_CAT_SELECT, launch_scan_counts(e->count, e->frame_offsets, e->d_small, T, n_dev, s));
-  PROF(ET_CAT_GATHER, launch_gather_tokens(e->X[cur], e->keep, e->frame_offsets, T, L, D, c.post_layernorm ? W + e->off_post_g : nullptr,
-                       c.post_layernorm ? W + e->off_post_b : nullptr, c.ln_eps, e->tokens, e->token_pos, n_dev, s));
+  PROF(ET_CAT_GATHER, launch_gather_tokens(e->X[cur], e->keep, e->count, e->frame_offsets, e->d_small, T, L, D,
+                       c.post_layernorm ? W + e->off_post_g : nullptr, c.post_layernorm ? W + e->off_post_b : nullptr,
+                       c.ln_eps, e->tokens, e->token_pos, n_dev, s));
   ET_CUDA(e, cudaMemcpyAsync(e->h_small, e->d_small, sizeof(int) * 16, cudaMemcpyDeviceToHost, s));
   ET_CUDA(e, cudaGetLastError());
   ET_CUDA(e, cudaStreamSynchronize(s));
@@ -395,7 +405,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     for (int layer = 0, m = 0; layer < c.num_layers; ++layer) {
       if (m < p->num_merge_layers && p->merge_layers[m] == layer) {
         const int n_out = e->h_small[2 + m];
-        wk[ET_CAT_SIMILARITY] += (double)n_in * dL * dD * 4.0 + 2.0 * (n_in - 1) * dL * 4.0;
+        wk[ET_CAT_SIMILARITY] += (double)n_in * dL * dD * 4.0;
         wk[ET_CAT_MERGE] += ((double)n_in + n_out) * dL * dD * 4.0;
         n_in = n_out; ++m;
       }
@@ -404,7 +414,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
       wk[ET_CAT_ATTENTION] += 4.0 * rows * dL * dD;
       wk[ET_CAT_LAYERNORM] += 2.0 * rows * dD * (4.0 + es);
     }
-    if (p->num_merge_layers == 0) wk[ET_CAT_SIMILARITY] += (double)N * dL * dD * 4.0 + 2.0 * (N - 1) * dL * 4.0;
+    if (p->num_merge_layers == 0) wk[ET_CAT_SIMILARITY] += (double)N * dL * dD * 4.0;
     wk[ET_CAT_SCORES] += 2.0 * N * dL * dL * dD;
     wk[ET_CAT_SELECT] += (double)N * dL * 5.0;
     wk[ET_CAT_GATHER] += 2.0 * n_tok * dD * 4.0;
@@ -481,6 +491,16 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   if ((st = dalloc(e, &e->w_blob, weights->count)) != ET_OK) return bail(st);
   if (cudaMemcpy(e->w_blob, weights->data, weights->count * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
     return bail(ET_ERR_CUDA);
+  {
+    int* flag = nullptr;
+    int bad = 0;
+    if ((st = dalloc(e, &flag, 1)) != ET_OK) return bail(st);
+    cudaMemset(flag, 0, sizeof(int));
+    ET_COUNT_LAUNCH();
+    find_nonfinite_kernel<<<148 * 8, 256>>>(e->w_blob, weights->count, flag);
+    if (cudaMemcpy(&bad, flag, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return bail(ET_ERR_CUDA);
+    if (bad) return bail(ET_ERR_WEIGHTS);
+  }
   const size_t es = e->bf ? 2 : 4;
   // ---- activations
 #define ET_A(ptr, bytes)                                                     \
@@ -493,7 +513,7 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   ET_A(e->Pm, rows * e->Kp * es); ET_A(e->Xn, rows * D * es); ET_A(e->QKV, rows * 3 * D * es);
   ET_A(e->O, rows * D * es); ET_A(e->Hm, rows * M * es);
   ET_A(e->lse, F * config->heads * L * 4); ET_A(e->score_partial, F * config->heads * L * 4);
-  ET_A(e->scores, rows * 4); ET_A(e->cosbuf, rows * 4); ET_A(e->simbuf, F * 4);
+  ET_A(e->scores, rows * 4); ET_A(e->simbuf, F * 4);
   for (int i = 0; i < 2; ++i) {
     ET_A(e->fl[i].n, 4); ET_A(e->fl[i].vid_off, (e->Vmax + 1) * 4); ET_A(e->fl[i].src_lo, F * 4);
     ET_A(e->fl[i].src_hi, F * 4); ET_A(e->fl[i].role, F);
@@ -504,7 +524,8 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
     ET_A(e->forced_seg[i], F); ET_A(e->forced_mrg[i], F);
   }
   ET_A(e->orig_vid_off, (e->Vmax + 1) * 4);
-  ET_A(e->dynamic, F); ET_A(e->keep, rows); ET_A(e->k_frame, F * 4); ET_A(e->w_frame, F * 4);
+  ET_A(e->dynamic, F); ET_A(e->keep, rows);
+  ET_A(e->sim_acc, (size_t)similarity_plan_words(e->Fmax) * 8);
   ET_A(e->video_k, e->Vmax * 4); ET_A(e->video_w, e->Vmax * 4); ET_A(e->count, F * 4);
   ET_A(e->frame_offsets, (F + 1) * 4); ET_A(e->token_pos, rows * 4); ET_A(e->tokens, rows * D * 4);
   ET_A(e->d_small, 16 * 4);
@@ -521,6 +542,7 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   // zero the activation buffers once: rows beyond the live count are read (never stored) by tile loads
   cudaMemset(e->Pm, 0, rows * e->Kp * es); cudaMemset(e->Xn, 0, rows * D * es); cudaMemset(e->O, 0, rows * D * es);
   cudaMemset(e->Hm, 0, rows * M * es); cudaMemset(e->QKV, 0, rows * 3 * D * es);
+  cudaMemset(e->sim_acc, 0, (size_t)similarity_plan_words(e->Fmax) * 8);
 
   if (e->bf) {
     // transposed bf16 copies of the dense weights ([out][in], K contiguous) + their tensor maps
@@ -691,7 +713,7 @@ et_status et_merge_plan(const float* sim_dev, const int* video_offsets_dev, int 
   a.trace = LayerTrace{sim_tr, ema_dev, seg_start_dev, merge_next_dev};
   a.alpha = ema_alpha; a.tau_seg = tau_seg; a.tau_merge = tau_merge; a.weighted = weighted_merge;
   a.allow_merge = 1; a.n_videos = V; a.status = status;
-  launch_merge_plan(a, s);
+  launch_merge_plan(a, n, s);
   cudaError_t err = cudaStreamSynchronize(s);
   cudaFree(scratch);
   return err == cudaSuccess ? ET_OK : ET_ERR_CUDA;
@@ -713,8 +735,7 @@ et_status et_select_tokens(const float* scores_dev, const unsigned char* dynamic
   if (!scores_dev || !dynamic_dev || !k_dev || !w_dev || !keep_dev || !count_dev) return ET_ERR_INVALID_ARG;
   if (window_mode < 0 || window_mode > 1) return ET_ERR_INVALID_ARG;
   if (N < 1 || L < 1 || L > 4096) return ET_ERR_SHAPE;
-  launch_select_tokens(scores_dev, dynamic_dev, k_dev, w_dev, N, L, 0, window_mode, keep_dev, count_dev, nullptr,
-                       (cudaStream_t)cuda_stream);
+  launch_select_tokens(scores_dev, dynamic_dev, k_dev, w_dev, N, L, window_mode, keep_dev, count_dev, (cudaStream_t)cuda_stream);
   ET_CUDA0(cudaGetLastError());
   return ET_OK;
 }
@@ -736,8 +757,8 @@ et_status et_gather_tokens(const float* x_dev, const unsigned char* keep_dev, in
   if (err == cudaSuccess) err = cudaStreamSynchronize(s);
   if (err != cudaSuccess) { cudaFree(scratch); return ET_ERR_CUDA; }
   if ((size_t)totals[1] > tokens_capacity_rows) { cudaFree(scratch); return ET_ERR_CAPACITY; }
-  launch_gather_tokens(x_dev, keep_dev, frame_offsets_dev, N, L, D, ln_g_dev, ln_b_dev, ln_eps, tokens_dev, token_pos_dev,
-                       nullptr, s);
+  launch_gather_tokens(x_dev, keep_dev, count, frame_offsets_dev, scratch, N, L, D, ln_g_dev, ln_b_dev, ln_eps, tokens_dev,
+                       token_pos_dev, nullptr, s);
   err = cudaStreamSynchronize(s);
   cudaFree(scratch);
   if (err != cudaSuccess) return ET_ERR_CUDA;

@@ -5,6 +5,9 @@
 
 namespace et {
 
+ET_DEBUG_STATUS_WORD
+ET_DEBUG_STATUS_READ(stage1_debug_status)
+
 // ---------------------------------------------------------------------------------------------
 // Token cosines.  One warp owns spatial position l over a run of consecutive frames: it keeps the
 // previous frame's row (and its squared norm) in registers, so every row of X is read from memory
@@ -12,6 +15,65 @@ namespace et {
 // Reductions: lane-local sums over a fixed chunk order, then a xor-shuffle tree -> bit-reproducible.
 // ---------------------------------------------------------------------------------------------
 constexpr int COS_RUN = 8;   // pairs per warp job
+
+// One job: position l over the pairs t0 .. t1-1 (frames t0 .. t1).  `is_cross(t)` says that frames t and t+1
+// belong to different videos: their cosine is never used, so it is not computed.  `emit(t, c)` receives the
+// cosine of pair t (same value in every lane).
+template <int NV, typename CrossFn, typename EmitFn>
+__device__ __forceinline__ void cos_run(const float* __restrict__ x, int l, int t0, int t1, int L, int D, int lane,
+                                        CrossFn is_cross, EmitFn emit) {
+  const int nvec = D >> 2;
+  const size_t frame_stride = (size_t)L * D;
+  const float4* row = reinterpret_cast<const float4*>(x + (size_t)t0 * frame_stride + (size_t)l * D);
+  float4 prev[NV], cur[NV];
+  float np = 0.f;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int i = lane + 32 * j;
+    prev[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  row = reinterpret_cast<const float4*>(x + (size_t)(t0 + 1) * frame_stride + (size_t)l * D);
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int i = lane + 32 * j;
+    cur[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int j = 0; j < NV; ++j)
+    np += (prev[j].x * prev[j].x + prev[j].y * prev[j].y) + (prev[j].z * prev[j].z + prev[j].w * prev[j].w);
+  np = warp_sum(np);
+  for (int t = t0; t < t1; ++t) {
+    // the row after next is requested before this pair is reduced, so that loads stay in flight
+    float4 nxt[NV];
+    if (t + 1 < t1) {
+      row = reinterpret_cast<const float4*>(x + (size_t)(t + 2) * frame_stride + (size_t)l * D);
+#pragma unroll
+      for (int j = 0; j < NV; ++j) {
+        const int i = lane + 32 * j;
+        nxt[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    float dot = 0.f, nc = 0.f;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      const float4 c = cur[j];
+      dot += (prev[j].x * c.x + prev[j].y * c.y) + (prev[j].z * c.z + prev[j].w * c.w);
+      nc += (c.x * c.x + c.y * c.y) + (c.z * c.z + c.w * c.w);
+    }
+    dot = warp_sum(dot);
+    nc = warp_sum(nc);
+    if (!is_cross(t)) emit(t, dot / fmaxf(sqrtf(np) * sqrtf(nc), 1e-8f));
+    np = nc;
+    if (t + 1 < t1) {
+#pragma unroll
+      for (int j = 0; j < NV; ++j) { prev[j] = cur[j]; cur[j] = nxt[j]; }
+    }
+  }
+}
+
+struct NoCross {
+  __device__ __forceinline__ bool operator()(int) const { return false; }
+};
 
 template <int NV>
 __global__ void __launch_bounds__(128)
@@ -22,57 +84,12 @@ token_cos_kernel(const float* __restrict__ x, float* __restrict__ cosbuf, int n_
   if (n_pairs <= 0) return;
   const int n_runs = (n_pairs + COS_RUN - 1) / COS_RUN;
   const int lane = threadIdx.x & 31;
-  const int nvec = D >> 2;
   const int warps_total = gridDim.x * (blockDim.x >> 5);
-  const size_t frame_stride = (size_t)L * D;
   for (int job = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); job < n_runs * L; job += warps_total) {
     const int l = job % L, run = job / L;
     const int t0 = run * COS_RUN, t1 = min(t0 + COS_RUN, n_pairs);
-    const float4* row = reinterpret_cast<const float4*>(x + (size_t)t0 * frame_stride + (size_t)l * D);
-    float4 prev[NV], cur[NV];
-    float np = 0.f;
-#pragma unroll
-    for (int j = 0; j < NV; ++j) {
-      const int i = lane + 32 * j;
-      prev[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    row = reinterpret_cast<const float4*>(x + (size_t)(t0 + 1) * frame_stride + (size_t)l * D);
-#pragma unroll
-    for (int j = 0; j < NV; ++j) {
-      const int i = lane + 32 * j;
-      cur[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int j = 0; j < NV; ++j)
-      np += (prev[j].x * prev[j].x + prev[j].y * prev[j].y) + (prev[j].z * prev[j].z + prev[j].w * prev[j].w);
-    np = warp_sum(np);
-    for (int t = t0; t < t1; ++t) {
-      // the row after next is requested before this pair is reduced, so that loads stay in flight
-      float4 nxt[NV];
-      if (t + 1 < t1) {
-        row = reinterpret_cast<const float4*>(x + (size_t)(t + 2) * frame_stride + (size_t)l * D);
-#pragma unroll
-        for (int j = 0; j < NV; ++j) {
-          const int i = lane + 32 * j;
-          nxt[j] = (i < nvec) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-      }
-      float dot = 0.f, nc = 0.f;
-#pragma unroll
-      for (int j = 0; j < NV; ++j) {
-        const float4 c = cur[j];
-        dot += (prev[j].x * c.x + prev[j].y * c.y) + (prev[j].z * c.z + prev[j].w * c.w);
-        nc += (c.x * c.x + c.y * c.y) + (c.z * c.z + c.w * c.w);
-      }
-      dot = warp_sum(dot);
-      nc = warp_sum(nc);
-      if (lane == 0) cosbuf[(size_t)t * L + l] = dot / fmaxf(sqrtf(np) * sqrtf(nc), 1e-8f);
-      np = nc;
-      if (t + 1 < t1) {
-#pragma unroll
-        for (int j = 0; j < NV; ++j) { prev[j] = cur[j]; cur[j] = nxt[j]; }
-      }
-    }
+    cos_run<NV>(x, l, t0, t1, L, D, lane, NoCross(),
+                [=](int t, float c) { if (lane == 0) cosbuf[(size_t)t * L + l] = c; });
   }
 }
 
@@ -94,17 +111,23 @@ void launch_token_cosines(const float* x, float* cos_scratch, int n_cap, int L, 
 #undef ET_COS
 }
 
-// sim[t] = (1/L) sum_l cos[t][l] for the pairs t < n - 1; one warp per pair, fixed order.
+// sim[t] = (1/L) sum_l cos[t][l]: lane-strided partial sums, then the xor-shuffle tree (fixed order).
+__device__ __forceinline__ float reduce_pair(const float* __restrict__ cos_row, int L, int lane) {
+  float acc = 0.f;
+  for (int l = lane; l < L; l += 32) acc += __ldcg(cos_row + l);
+  acc = warp_sum(acc);
+  return acc / (float)L;
+}
+
+// one warp per pair t < n - 1
 __global__ void reduce_cos_kernel(const float* __restrict__ cosbuf, float* __restrict__ sim, int n_cap, int L,
                                   const int* __restrict__ n_frames_dev) {
   const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
   const int lane = threadIdx.x & 31;
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (t >= n - 1) return;
-  float acc = 0.f;
-  for (int l = lane; l < L; l += 32) acc += cosbuf[(size_t)t * L + l];
-  acc = warp_sum(acc);
-  if (lane == 0) sim[t] = acc / (float)L;
+  const float v = reduce_pair(cosbuf + (size_t)t * L, L, lane);
+  if (lane == 0) sim[t] = v;
 }
 
 void launch_reduce_cosines(const float* cos_scratch, float* sim, int n_cap, int L, const int* n_frames_dev,
@@ -120,132 +143,288 @@ void launch_reduce_cosines(const float* cos_scratch, float* sim, int n_cap, int 
 // bookkeeping of the next frame list.  Decision arithmetic is double, comparisons are the
 // paper's strict inequalities.
 // ---------------------------------------------------------------------------------------------
-__global__ void merge_plan_kernel(PlanArgs a) {
-  extern __shared__ int sh_count[];     // [n_videos + 1] output frames per video, then their scan
+constexpr int PLAN_STAGE_FRAMES = 2048;     // lists up to this length are planned out of shared memory
+static inline size_t plan_smem_bytes(int n_videos, int n_cap) {
+  return sizeof(int) * (n_videos + 1) + (size_t)min(n_cap, PLAN_STAGE_FRAMES) * (2 * sizeof(float) + 2 * sizeof(int) + 1);
+}
+
+// Per-frame flag byte while the plan is being made
+enum : unsigned char { PF_START = 1, PF_MERGE = 2, PF_LAST = 4, PF_FIRST = 8 };
+
+// The plan of one merge layer, executed by ONE warp (lane = 0..31).  Shared memory: sh_count [n_videos + 1] ints
+// followed by the staging area for `stage_frames` frames (similarity, EMA, source range, flag byte).
+//   phase A, a lane per video, frames in order: the EMA recurrence of Eq. 1 with its restarts, and the pairing of
+//            Eq. 2 inside each segment, are chains in which a step depends on the decision before it.  They only
+//            touch the staged arrays (a chain of reads from global memory would cost a memory latency per frame);
+//   phase B, a lane per frame: everything that depends on one frame and its neighbour -- the output index (a prefix
+//            sum of "this frame opens an output frame" by ballot / popc), the Eq. 3 weights, the source ranges and
+//            roles of the next list, the trace.
+// Lists longer than the staging area work on the global arrays (the trace arrays double as working storage).
+// Similarities are read past the L1 (other SMs may have written them during the same kernel).
+// Copies the list's similarities and source ranges into the staging area (any number of threads; the caller
+// synchronises them before merge_plan_body runs).  Nothing is staged when the list does not fit.
+__device__ __forceinline__ void merge_plan_stage(const PlanArgs& a, int tid, int nthr, int* sh_count, int stage_frames) {
+  const int n = *a.cur.n;
+  if (n > stage_frames) return;
+  float* const st_sim = reinterpret_cast<float*>(sh_count + a.n_videos + 1);
+  int* const st_lo = reinterpret_cast<int*>(st_sim + 2 * stage_frames);
+  int* const st_hi = st_lo + stage_frames;
+  for (int t = tid; t < n; t += nthr) {
+    st_sim[t] = __ldcg(a.sim + t);
+    st_lo[t] = a.cur.src_lo[t];
+    st_hi[t] = a.cur.src_hi[t];
+  }
+}
+
+__device__ void merge_plan_body(const PlanArgs& a, int lane, int* sh_count, int stage_frames) {
   const int V = a.n_videos;
   const int n = *a.cur.n;
   const bool forced = a.forced_seg_start != nullptr;
-  if (forced && threadIdx.x == 0 && a.forced_n_in != n) atomicExch(a.status, (int)DS_FORCED_MISMATCH);
+  if (forced && lane == 0 && a.forced_n_in != n) atomicExch(a.status, (int)DS_FORCED_MISMATCH);
   const bool use_forced = forced && a.forced_n_in == n;
-  unsigned char* const f_start = a.trace.seg_start;   // flags of the INPUT list (also the trace)
-  unsigned char* const f_merge = a.trace.merge_next;
+  const bool staged = n <= stage_frames;
+  float* const st_sim = reinterpret_cast<float*>(sh_count + V + 1);
+  float* const st_ema = st_sim + stage_frames;
+  int* const st_lo = reinterpret_cast<int*>(st_ema + stage_frames);
+  int* const st_hi = st_lo + stage_frames;
+  unsigned char* const st_flag = reinterpret_cast<unsigned char*>(st_hi + stage_frames);
+  float* const ema = staged ? st_ema : a.trace.ema;
+  unsigned char* const flag = staged ? st_flag : a.trace.seg_start;
+  auto sim_at = [&](int t) -> float { return staged ? st_sim[t] : __ldcg(a.sim + t); };
+  auto lo_at = [&](int t) -> int { return staged ? st_lo[t] : a.cur.src_lo[t]; };
+  auto hi_at = [&](int t) -> int { return staged ? st_hi[t] : a.cur.src_hi[t]; };
 
-  // Pass 1 (per video): Eq. 1 segmentation, Eq. 2 pairing, count of output frames.
-  for (int v = threadIdx.x; v < V; v += blockDim.x) {
+  // ---- phase A: per video, in frame order
+  for (int v = lane; v < V; v += 32) {
     const int g0 = a.cur.vid_off[v], g1 = a.cur.vid_off[v + 1];
     double prev = 0.0;
     bool have_prev = false;
-    for (int t = g0; t < g1; ++t) {
-      unsigned char start = 1;
+    for (int t = g0; t < g1; ++t) {                    // Eq. 1
+      unsigned char f = PF_START;
       float ema_out = 0.f;
       if (t > g0) {
-        const double s = (double)a.sim[t - 1];
+        const double s = (double)sim_at(t - 1);
         // explicit roundings: no fused multiply-add, so the value is the same as a plain host evaluation
         const double cur = have_prev ? __dadd_rn(__dmul_rn(a.alpha, s), __dmul_rn(1.0 - a.alpha, prev)) : s;
         ema_out = (float)cur;
-        start = use_forced ? (a.forced_seg_start[t] ? 1 : 0) : (cur < a.tau_seg ? 1 : 0);
+        const bool start = use_forced ? (a.forced_seg_start[t] != 0) : (cur < a.tau_seg);
+        f = start ? PF_START : 0;
         if (start) have_prev = false;
         else { prev = cur; have_prev = true; }
       }
-      f_start[t] = start;
-      a.trace.ema[t] = ema_out;
-      a.trace.sim[t] = (t < g1 - 1) ? a.sim[t] : 0.f;
-      f_merge[t] = 0;
+      if (t == g0) f |= PF_FIRST;
+      if (t == g1 - 1) f |= PF_LAST;
+      flag[t] = f;
+      ema[t] = ema_out;
     }
+    int out = g1 - g0;
     if (a.allow_merge && use_forced) {
+      bool prev_merged = false;
       for (int t = g0; t < g1; ++t) {
         bool m = a.forced_merge_next[t] != 0;
-        if (m && (t + 1 >= g1 || (t > g0 && f_merge[t - 1]))) { m = false; atomicExch(a.status, (int)DS_FORCED_MISMATCH); }
-        f_merge[t] = m ? 1 : 0;
+        if (m && (t + 1 >= g1 || prev_merged)) { m = false; atomicExch(a.status, (int)DS_FORCED_MISMATCH); }
+        if (m) { flag[t] |= PF_MERGE; --out; }
+        prev_merged = m;
       }
-    } else if (a.allow_merge) {
+    } else if (a.allow_merge) {                        // Eq. 2 inside each segment
       int seg_a = g0;
       while (seg_a < g1) {
-        int seg_b = seg_a;                       // last frame of the segment
-        while (seg_b + 1 < g1 && f_start[seg_b + 1] == 0) ++seg_b;
+        int seg_b = seg_a;                             // last frame of the segment
+        while (seg_b + 1 < g1 && !(flag[seg_b + 1] & PF_START)) ++seg_b;
         const int k = seg_b - seg_a;
         int i = 1;
-        while (i <= k - 1) {                     // middle frames g_1 .. g_{k-1}
+        while (i <= k - 2) {                           // both frames of a pair are middle frames g_1 .. g_{k-1}
           const int t = seg_a + i;
-          bool m = false;
-          if (i <= k - 2) {                      // both frames of the pair are middle frames
-            const double ci = (double)a.sim[t], cn = (double)a.sim[t + 1];
-            m = (ci > a.tau_merge) && (ci > cn);
-          }
-          f_merge[t] = m ? 1 : 0;
+          const double ci = (double)sim_at(t), cn = (double)sim_at(t + 1);
+          const bool m = (ci > a.tau_merge) && (ci > cn);
+          if (m) { flag[t] |= PF_MERGE; --out; }
           i += m ? 2 : 1;
         }
         seg_a = seg_b + 1;
       }
     }
-    int out = 0;
-    for (int t = g0; t < g1; t += f_merge[t] ? 2 : 1) ++out;
     sh_count[v] = out;
   }
-  __syncthreads();
-
-  if (!a.allow_merge) {   // segmentation only: roles of the unchanged list
-    for (int v = threadIdx.x; v < V; v += blockDim.x) {
-      const int g0 = a.cur.vid_off[v], g1 = a.cur.vid_off[v + 1];
-      for (int t = g0; t < g1; ++t) {
-        const bool s0 = f_start[t] != 0;
-        const bool s1 = (t + 1 >= g1) || f_start[t + 1] != 0;
-        a.cur.role[t] = s0 ? (s1 ? 3 : 0) : (s1 ? 2 : 1);
-      }
-    }
-    if (threadIdx.x == 0 && a.n_hist_slot) *a.n_hist_slot = n;
-    return;
-  }
-
-  if (threadIdx.x == 0) {
+  __syncwarp();
+  if (lane == 0) {                                     // offsets of the next list
     int acc = 0;
     for (int v = 0; v < V; ++v) { const int c = sh_count[v]; sh_count[v] = acc; acc += c; }
     sh_count[V] = acc;
   }
-  __syncthreads();
+  __syncwarp();
 
-  // Pass 2 (per video): emit the plan and the metadata of the next list, indexed by output frame.
-  for (int v = threadIdx.x; v < V; v += blockDim.x) {
-    const int g0 = a.cur.vid_off[v], g1 = a.cur.vid_off[v + 1];
-    int j = sh_count[v];
-    int t = g0;
-    while (t < g1) {
-      const bool mrg = f_merge[t] != 0;
+  // ---- phase B: per frame
+  int carry = 0;                                       // output frames before this chunk of 32 input frames
+  for (int base = 0; base < n; base += 32) {
+    const int t = base + lane;
+    const bool live = t < n;
+    const unsigned char f = live ? flag[t] : 0;
+    const unsigned char fp = (live && t > 0) ? flag[t - 1] : 0;
+    const unsigned char fn = (live && t + 1 < n) ? flag[t + 1] : 0;
+    const bool second = !(f & PF_FIRST) && (fp & PF_MERGE);      // the second frame of a merged pair
+    const bool opens = live && !second;
+    const unsigned m = __ballot_sync(0xffffffffu, opens);
+    const int j = carry + __popc(m & ((1u << lane) - 1u));
+    carry += __popc(m);
+    if (!live) continue;
+    const bool last = (f & PF_LAST) != 0;
+    const bool mrg = (f & PF_MERGE) != 0;
+    if (a.allow_merge && opens) {
+      ET_CHECK(j >= 0 && j < n && (!mrg || !last), continue);
       if (mrg) {
-        const double ca = (double)a.sim[t];
-        const double cb = (t + 1 < g1 - 1) ? (double)a.sim[t + 1] : 0.0;   // similarity to the following frame
+        const double ca = (double)sim_at(t);
+        const double cb = (fn & PF_LAST) ? 0.0 : (double)sim_at(t + 1);     // similarity to the following frame
         const double den = ca + cb;
         float wa = 0.5f, wb = 0.5f;
         if (a.weighted && den > 1e-6) { wa = (float)(ca / den); wb = (float)(cb / den); }
         a.plan.src_a[j] = t; a.plan.src_b[j] = t + 1;
         a.plan.w_a[j] = wa;  a.plan.w_b[j] = wb;
-        a.nxt.src_lo[j] = a.cur.src_lo[t];
-        a.nxt.src_hi[j] = a.cur.src_hi[t + 1];
+        a.nxt.src_lo[j] = lo_at(t);
+        a.nxt.src_hi[j] = hi_at(t + 1);
         a.nxt.role[j] = 1;
       } else {
-        const bool s0 = f_start[t] != 0;
-        const bool s1 = (t + 1 >= g1) || f_start[t + 1] != 0;
+        const bool s0 = (f & PF_START) != 0;
+        const bool s1 = last || (fn & PF_START);
         a.plan.src_a[j] = t; a.plan.src_b[j] = -1;
         a.plan.w_a[j] = 1.f; a.plan.w_b[j] = 0.f;
-        a.nxt.src_lo[j] = a.cur.src_lo[t];
-        a.nxt.src_hi[j] = a.cur.src_hi[t];
+        a.nxt.src_lo[j] = lo_at(t);
+        a.nxt.src_hi[j] = hi_at(t);
         a.nxt.role[j] = s0 ? (s1 ? 3 : 0) : (s1 ? 2 : 1);
       }
-      ++j;
-      t += mrg ? 2 : 1;
     }
+    if (!a.allow_merge) {                              // segmentation only: roles of the unchanged list
+      const bool s0 = (f & PF_START) != 0;
+      const bool s1 = last || (fn & PF_START);
+      a.cur.role[t] = s0 ? (s1 ? 3 : 0) : (s1 ? 2 : 1);
+    }
+    a.trace.sim[t] = last ? 0.f : sim_at(t);
+    if (staged) a.trace.ema[t] = ema[t];
+    a.trace.merge_next[t] = mrg ? 1 : 0;
   }
-  for (int v = threadIdx.x; v <= V; v += blockDim.x) a.nxt.vid_off[v] = sh_count[v];
-  if (threadIdx.x == 0) {
+  __syncwarp();                                        // every neighbour's flag has been read
+  for (int t = lane; t < n; t += 32) a.trace.seg_start[t] = (flag[t] & PF_START) ? 1 : 0;
+  if (!a.allow_merge) {
+    if (lane == 0 && a.n_hist_slot) *a.n_hist_slot = n;
+    return;
+  }
+  for (int v = lane; v <= V; v += 32) a.nxt.vid_off[v] = sh_count[v];
+  if (lane == 0) {
     *a.nxt.n = sh_count[V];
     if (a.n_hist_slot) *a.n_hist_slot = sh_count[V];
   }
 }
 
-void launch_merge_plan(const PlanArgs& a, cudaStream_t s) {
+__global__ void merge_plan_kernel(PlanArgs a, int stage_frames) {
+  extern __shared__ int sh_plan_count[];
+  merge_plan_stage(a, threadIdx.x, blockDim.x, sh_plan_count, stage_frames);
+  __syncthreads();
+  if (threadIdx.x < 32) merge_plan_body(a, threadIdx.x, sh_plan_count, stage_frames);
+}
+
+void launch_merge_plan(const PlanArgs& a, int n_cap, cudaStream_t s) {
   ET_COUNT_LAUNCH();
-  const int threads = min(1024, max(32, ((a.n_videos + 31) / 32) * 32));
-  merge_plan_kernel<<<1, threads, sizeof(int) * (a.n_videos + 1), s>>>(a);
+  merge_plan_kernel<<<1, 128, plan_smem_bytes(a.n_videos, n_cap), s>>>(a, min(n_cap, PLAN_STAGE_FRAMES));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Similarities and plan in ONE launch (the encoder's path).  Jobs are the (run of 8 pairs, position) items of
+// token_cos_kernel.  The mean over positions is accumulated without any scratch array and without any order:
+// every cosine is scaled by 2^32, rounded to an integer and added to the pair's 64-bit accumulator with an atomic
+// add.  Integer addition is exact and commutative, so the result does not depend on the order of arrival (bit-
+// reproducible), and the rounding step (2^-32 per position) is far below the fp32 rounding of the cosine itself.
+// Nobody waits for anybody: a block that has finished all its jobs takes one ticket; the block that takes the last
+// ticket turns the accumulators into similarities (resetting them for the next launch) and runs the plan
+// (Eq. 1-2, Eq. 3 weights, next list).  Pairs that straddle two videos are not computed.
+// ---------------------------------------------------------------------------------------------
+constexpr double SIM_FIXED_ONE = 4294967296.0;     // 2^32
+// A pair's sum is spread over SIM_SLOTS accumulators (slot = position mod SIM_SLOTS, n_cap words apart): all warps
+// work on the same few pairs at the same time, and thousands of atomic adds to one address queue up in one L2 slice.
+constexpr int SIM_SLOTS = 16;
+
+template <int NV>
+__global__ void __launch_bounds__(128) similarity_plan_kernel(SimPlanArgs a) {
+  extern __shared__ int sh_plan[];      // used only by the block that runs the plan
+  __shared__ unsigned sh_last;
+  const int n = min(*a.n_frames_dev, a.n_cap);
+  const int n_pairs = n - 1;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+  const int stage = min(a.n_cap, PLAN_STAGE_FRAMES);
+  if (n_pairs <= 0) {                   // single frame: nothing to compare, the plan still sets roles and counts
+    if (blockIdx.x == 0) {
+      merge_plan_stage(a.plan, threadIdx.x, blockDim.x, sh_plan, stage);
+      __syncthreads();
+      if (warp == 0) merge_plan_body(a.plan, lane, sh_plan, stage);
+    }
+    return;
+  }
+  const int n_runs = (n_pairs + COS_RUN - 1) / COS_RUN;
+  const int n_jobs = n_runs * a.L;
+  if (blockIdx.x * wpb >= n_jobs) return;               // blocks without a job take no ticket
+  const int warps_total = gridDim.x * wpb;
+  const int* vo = a.vid_off;
+  int v = 0;                            // video of the current frame; jobs of a warp come in ascending frame order
+  for (int job = blockIdx.x * wpb + warp; job < n_jobs; job += warps_total) {
+    const int l = job % a.L, run = job / a.L;
+    const int t0 = run * COS_RUN, t1 = min(t0 + COS_RUN, n_pairs);
+    ET_CHECK(t0 >= 0 && t1 <= a.n_cap - 1 && t0 < vo[a.n_videos], continue);
+    unsigned cross = 0;                 // bit q: frames t0+q and t0+q+1 belong to different videos
+    for (int t = t0; t < t1; ++t) {
+      while (vo[v + 1] <= t) ++v;
+      if (t + 1 == vo[v + 1]) cross |= 1u << (t - t0);
+    }
+    auto is_cross = [cross, t0](int t) { return ((cross >> (t - t0)) & 1u) != 0; };
+    unsigned long long* acc = a.acc + (size_t)(l % SIM_SLOTS) * a.n_cap;
+    cos_run<NV>(a.x, l, t0, t1, a.L, a.D, lane, is_cross, [=](int t, float c) {
+      if (lane == 0) atomicAdd(acc + t, (unsigned long long)__double2ll_rn((double)c * SIM_FIXED_ONE));
+    });
+  }
+  if (lane == 0) __threadfence();       // this warp's additions before the block's ticket
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned blocks_with_jobs = (unsigned)min((long long)gridDim.x, ((long long)n_jobs + wpb - 1) / wpb);
+    sh_last = atomicAdd(a.done, 1u) == blocks_with_jobs - 1u ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!sh_last) return;
+  // the last block: accumulators -> similarities (and back to zero for the next launch), then the plan
+  __threadfence();
+  for (int t = threadIdx.x; t < n_pairs; t += blockDim.x) {
+    unsigned long long part[SIM_SLOTS];
+#pragma unroll
+    for (int q = 0; q < SIM_SLOTS; ++q) part[q] = __ldcg(a.acc + (size_t)q * a.n_cap + t);   // the adds happened at the L2
+    unsigned long long sum = 0;
+#pragma unroll
+    for (int q = 0; q < SIM_SLOTS; ++q) {
+      sum += part[q];
+      a.acc[(size_t)q * a.n_cap + t] = 0ull;
+    }
+    a.sim[t] = (float)((double)(long long)sum / (SIM_FIXED_ONE * (double)a.L));      // the mean, rounded once
+  }
+  if (threadIdx.x == 0) *a.done = 0u;
+  __threadfence();
+  __syncthreads();
+  merge_plan_stage(a.plan, threadIdx.x, blockDim.x, sh_plan, stage);
+  __syncthreads();
+  if (warp == 0) merge_plan_body(a.plan, lane, sh_plan, stage);
+}
+
+int similarity_plan_words(int n_cap) { return SIM_SLOTS * n_cap + 1; }
+
+void launch_similarity_plan(const SimPlanArgs& a, cudaStream_t s) {
+  const int runs = max(1, cdiv(max(a.n_cap - 1, 1), COS_RUN));
+  const int blocks = max(1, min(cdiv((long long)runs * a.L, 4), 148 * 16));
+  const int need = cdiv(a.D / 4, 32);
+  const size_t smem = plan_smem_bytes(a.n_videos, a.n_cap);
+  ET_COUNT_LAUNCH();
+#define ET_SP(NV) similarity_plan_kernel<NV><<<blocks, 128, smem, s>>>(a)
+  if (need <= 1) ET_SP(1);
+  else if (need <= 2) ET_SP(2);
+  else if (need <= 4) ET_SP(4);
+  else if (need <= 6) ET_SP(6);
+  else if (need <= 9) ET_SP(9);
+  else if (need <= 12) ET_SP(12);
+  else ET_SP(16);
+#undef ET_SP
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -258,6 +437,7 @@ merge_frames_kernel(const float4* __restrict__ x, float4* __restrict__ y, int fr
   const int j = blockIdx.y;
   if (j >= *n_out_dev) return;
   const int sa = plan.src_a[j], sb = plan.src_b[j];
+  ET_CHECK(sa >= 0 && sa < (int)gridDim.y && sb >= -1 && sb < (int)gridDim.y, return);
   const float4* xa = x + (size_t)sa * frame_vec4;
   float4* yo = y + (size_t)j * frame_vec4;
   if (sb < 0) {

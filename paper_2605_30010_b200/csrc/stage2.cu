@@ -5,41 +5,8 @@
 
 namespace et {
 
-// ---------------------------------------------------------------------------------------------
-// Per-video amounts and per-frame flags.  One thread per video computes k (Eq. 5 read as a
-// per-frame token count) and the window width w (Eq. 6) in double, with the same expression
-// order as a plain host evaluation; then all threads fill the per-frame arrays.
-// ---------------------------------------------------------------------------------------------
-__global__ void select_setup_kernel(SelectSetupArgs a) {
-  const int V = a.n_videos;
-  for (int v = threadIdx.x; v < V; v += blockDim.x) {
-    const int N = a.fl.vid_off[v + 1] - a.fl.vid_off[v];
-    const int B = a.orig_vid_off[v + 1] - a.orig_vid_off[v];
-    int k;
-    if (a.retain_mode == 1) k = (int)floor(a.retain * (double)B * (double)a.L / (double)max(N, 1) + 1e-9);
-    else k = (int)floor(a.retain * (double)a.L + 1e-9);
-    k = max(1, min(a.L, k));
-    const int w = max(1, a.L / k);      // reported in both window modes; mode 1 cuts k near-equal windows instead
-    a.video_k[v] = k;
-    a.video_w[v] = w;
-  }
-  __syncthreads();
-  for (int v = 0; v < V; ++v) {
-    const int g0 = a.fl.vid_off[v], g1 = a.fl.vid_off[v + 1];
-    for (int t = g0 + threadIdx.x; t < g1; t += blockDim.x) {
-      const bool dyn = a.fl.role[t] != 1;
-      a.dynamic[t] = dyn ? 1 : 0;
-      a.k_frame[t] = a.video_k[v];
-      a.w_frame[t] = a.video_w[v];
-    }
-  }
-}
-
-void launch_select_setup(const SelectSetupArgs& a, int n_cap, cudaStream_t s) {
-  (void)n_cap;
-  ET_COUNT_LAUNCH();
-  select_setup_kernel<<<1, 256, 0, s>>>(a);
-}
+ET_DEBUG_STATUS_WORD
+ET_DEBUG_STATUS_READ(stage2_debug_status)
 
 // ---------------------------------------------------------------------------------------------
 // Selection: one CTA per frame, scores in shared memory.
@@ -53,26 +20,11 @@ void launch_select_setup(const SelectSetupArgs& a, int n_cap, cudaStream_t s) {
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ float nan_to_lowest(float v) { return v != v ? -INFINITY : v; }
 
-__global__ void __launch_bounds__(256)
-select_tokens_kernel(const float* __restrict__ scores, const unsigned char* __restrict__ dynamic,
-                     const int* __restrict__ k_frame, const int* __restrict__ w_frame, int n_cap, int L,
-                     int selection_all, int window_mode, unsigned char* __restrict__ keep, int* __restrict__ count,
-                     const int* __restrict__ n_frames_dev) {
-  extern __shared__ float sh_a[];
-  const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
-  const int f = blockIdx.x;
-  if (f >= n) return;
-  const float* a = scores + (size_t)f * L;
-  unsigned char* kp = keep + (size_t)f * L;
-  if (selection_all) {
-    for (int j = threadIdx.x; j < L; j += blockDim.x) kp[j] = 1;
-    if (threadIdx.x == 0) count[f] = L;
-    return;
-  }
-  for (int j = threadIdx.x; j < L; j += blockDim.x) sh_a[j] = nan_to_lowest(a[j]);
-  __syncthreads();
-  const int k = max(1, min(k_frame[f], L));
-  if (dynamic[f]) {
+// The frame's scores are in sh_a (NaN already mapped); writes the mask row and returns the kept count (uniform).
+__device__ __forceinline__ int select_frame(const float* sh_a, int L, bool dyn, int k_in, int w_in, int window_mode,
+                                            unsigned char* __restrict__ kp) {
+  const int k = max(1, min(k_in, L));
+  if (dyn) {
     for (int j = threadIdx.x; j < L; j += blockDim.x) {
       const float aj = sh_a[j];
       int rank = 0;
@@ -82,31 +34,96 @@ select_tokens_kernel(const float* __restrict__ scores, const unsigned char* __re
       }
       kp[j] = rank < k ? 1 : 0;
     }
-    if (threadIdx.x == 0) count[f] = k;       // the order is total, so exactly k ranks are below k
-  } else {
-    const int w = max(1, min(w_frame[f], L));
-    const int M = window_mode == 1 ? k : (L + w - 1) / w;
-    for (int j = threadIdx.x; j < L; j += blockDim.x) kp[j] = 0;
-    __syncthreads();
-    for (int m = threadIdx.x; m < M; m += blockDim.x) {
-      const int lo = window_mode == 1 ? (int)(((long long)m * L) / k) : m * w;
-      const int hi = window_mode == 1 ? (int)(((long long)(m + 1) * L) / k) : min(lo + w, L);
-      int best = lo;
-      for (int j = lo + 1; j < hi; ++j)
-        if (sh_a[j] > sh_a[best]) best = j;
-      kp[best] = 1;
-    }
-    if (threadIdx.x == 0) count[f] = M;       // windows are disjoint and non-empty: one byte set per window
+    return k;                                  // the order is total, so exactly k ranks are below k
   }
+  const int w = max(1, min(w_in, L));
+  const int M = window_mode == 1 ? k : (L + w - 1) / w;
+  for (int j = threadIdx.x; j < L; j += blockDim.x) kp[j] = 0;
+  __syncthreads();
+  for (int m = threadIdx.x; m < M; m += blockDim.x) {
+    const int lo = window_mode == 1 ? (int)(((long long)m * L) / k) : m * w;
+    const int hi = window_mode == 1 ? (int)(((long long)(m + 1) * L) / k) : min(lo + w, L);
+    ET_CHECK(lo >= 0 && lo < hi && hi <= L, continue);
+    int best = lo;
+    for (int j = lo + 1; j < hi; ++j)
+      if (sh_a[j] > sh_a[best]) best = j;
+    kp[best] = 1;
+  }
+  return M;                                    // windows are disjoint and non-empty: one byte set per window
+}
+
+// amounts given per frame (the single-step entry point)
+__global__ void __launch_bounds__(256)
+select_tokens_kernel(const float* __restrict__ scores, const unsigned char* __restrict__ dynamic,
+                     const int* __restrict__ k_frame, const int* __restrict__ w_frame, int n_cap, int L,
+                     int window_mode, unsigned char* __restrict__ keep, int* __restrict__ count) {
+  extern __shared__ float sh_a[];
+  const int f = blockIdx.x;
+  if (f >= n_cap) return;
+  const float* a = scores + (size_t)f * L;
+  for (int j = threadIdx.x; j < L; j += blockDim.x) sh_a[j] = nan_to_lowest(a[j]);
+  __syncthreads();
+  const int c = select_frame(sh_a, L, dynamic[f] != 0, k_frame[f], w_frame[f], window_mode, keep + (size_t)f * L);
+  if (threadIdx.x == 0) count[f] = c;
+}
+
+// The encoder's path: one CTA per frame finds its video, derives the video's amounts (Eq. 5 read as a per-frame
+// token count k, window width w of Eq. 6; double arithmetic in the expression order of a plain host evaluation),
+// the frame's dynamic flag (head / tail of its segment) and the mask, in one launch.
+__global__ void __launch_bounds__(256) select_video_tokens_kernel(SelectArgs a) {
+  extern __shared__ float sh_a[];
+  __shared__ int sh_v;
+  const int n = min(*a.fl.n, a.n_cap);
+  const int f = blockIdx.x;
+  if (f >= n) return;
+  if (threadIdx.x == 0) {
+    int lo = 0, hi = a.n_videos;               // invariant: vid_off[lo] <= f < vid_off[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (a.fl.vid_off[mid] <= f) lo = mid; else hi = mid;
+    }
+    sh_v = lo;
+  }
+  const float* sc = a.scores + (size_t)f * a.L;
+  for (int j = threadIdx.x; j < a.L; j += blockDim.x) sh_a[j] = nan_to_lowest(sc[j]);
+  __syncthreads();
+  const int v = sh_v, L = a.L;
+  ET_CHECK(v >= 0 && v < a.n_videos && a.fl.vid_off[v] <= f && f < a.fl.vid_off[v + 1], return);
+  const int N = a.fl.vid_off[v + 1] - a.fl.vid_off[v];
+  const int B = a.orig_vid_off[v + 1] - a.orig_vid_off[v];
+  int k;
+  if (a.retain_mode == 1) k = (int)floor(a.retain * (double)B * (double)L / (double)max(N, 1) + 1e-9);
+  else k = (int)floor(a.retain * (double)L + 1e-9);
+  k = max(1, min(L, k));
+  const int w = max(1, L / k);                 // reported in both window modes; mode 1 cuts k near-equal windows
+  const bool dyn = a.fl.role[f] != 1;
+  if (threadIdx.x == 0) {
+    a.dynamic[f] = dyn ? 1 : 0;
+    if (f == a.fl.vid_off[v]) { a.video_k[v] = k; a.video_w[v] = w; }
+  }
+  if (a.mask_given) return;                    // the mask comes from the caller: only flags and amounts
+  unsigned char* kp = a.keep + (size_t)f * L;
+  if (a.selection == 0) {
+    for (int j = threadIdx.x; j < L; j += blockDim.x) kp[j] = 1;
+    if (threadIdx.x == 0) a.count[f] = L;
+    return;
+  }
+  const int c = select_frame(sh_a, L, dyn || a.selection >= 2, k, w, a.window_mode, kp);
+  if (threadIdx.x == 0) a.count[f] = c;
+}
+
+void launch_select_video_tokens(const SelectArgs& a, cudaStream_t s) {
+  if (a.n_cap <= 0) return;
+  ET_COUNT_LAUNCH();
+  select_video_tokens_kernel<<<a.n_cap, 256, sizeof(float) * a.L, s>>>(a);
 }
 
 void launch_select_tokens(const float* scores, const unsigned char* dynamic, const int* k_frame, const int* w_frame,
-                          int n_cap, int L, int selection_all, int window_mode, unsigned char* keep, int* count,
-                          const int* n_frames_dev, cudaStream_t s) {
+                          int n_cap, int L, int window_mode, unsigned char* keep, int* count, cudaStream_t s) {
   if (n_cap <= 0) return;
   ET_COUNT_LAUNCH();
-  select_tokens_kernel<<<n_cap, 256, sizeof(float) * L, s>>>(scores, dynamic, k_frame, w_frame, n_cap, L,
-                                                             selection_all, window_mode, keep, count, n_frames_dev);
+  select_tokens_kernel<<<n_cap, 256, sizeof(float) * L, s>>>(scores, dynamic, k_frame, w_frame, n_cap, L, window_mode,
+                                                             keep, count);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -217,41 +234,73 @@ void launch_scan_counts(const int* count, int* frame_offsets, int* totals, int n
 }
 
 // ---------------------------------------------------------------------------------------------
-// Gather (Eq. 7) with optional LayerNorm.  grid = (slices, frames).  Each CTA recomputes the
-// frame's compaction map by a warp-level prefix sum over ballots of the keep bytes (32 positions
-// per step, carry in a register), then its warps move their share of the kept rows:
-// warp-per-row, row in registers, LayerNorm statistics by shuffles.
+// Gather (Eq. 7) with optional LayerNorm.  grid = (slices, frames).  Each CTA sums the counts of the
+// frames before its own (the frame's first output row; the CTA of slice 0 records it, and the last
+// frame's also records the totals) and recomputes the frame's compaction map by a warp-level prefix
+// sum: every warp ballots the keep bytes of its eighth of the positions, the warps' totals are
+// scanned through shared memory, and popc of the ballot below a lane gives each kept position its
+// rank; then the warps move their share of the kept rows: warp-per-row, row in registers, LayerNorm
+// statistics by shuffles.
 // ---------------------------------------------------------------------------------------------
 
 template <int NV>
 __global__ void __launch_bounds__(256)
-gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restrict__ keep,
-                     const int* __restrict__ frame_offsets, int n_cap, int L, int D, const float* __restrict__ ln_g,
-                     const float* __restrict__ ln_b, float eps, float* __restrict__ tokens,
+gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restrict__ keep, const int* __restrict__ count,
+                     int* __restrict__ frame_offsets, int* __restrict__ totals, int n_cap, int L, int D,
+                     const float* __restrict__ ln_g, const float* __restrict__ ln_b, float eps, float* __restrict__ tokens,
                      int* __restrict__ token_pos, const int* __restrict__ n_frames_dev) {
   extern __shared__ unsigned short sh_pos[];   // [L] position of the r-th kept token of this frame
-  __shared__ int sh_kept;
+  __shared__ int sh_before[8], sh_wkept[8];
   const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
   const int f = blockIdx.y;
   if (f >= n) return;
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nwarps = blockDim.x >> 5;   // 8 warps
   const unsigned char* kp = keep + (size_t)f * L;
-  if (wid == 0) {
-    int carry = 0;
-    for (int base = 0; base < L; base += 32) {
-      const int j = base + lane;
-      const bool k = j < L && kp[j] != 0;
-      const unsigned m = __ballot_sync(0xffffffffu, k);
-      if (k) sh_pos[carry + __popc(m & ((1u << lane) - 1u))] = (unsigned short)j;
-      carry += __popc(m);
-    }
-    if (lane == 0) sh_kept = carry;
+  // first output row of this frame: the counts of the frames before it (integer sum: any order gives the same)
+  int before = 0;
+  for (int g = threadIdx.x; g < f; g += blockDim.x) before += count[g];
+  // compaction map: warp w owns the positions [w*chunk, (w+1)*chunk); ballots of its keep bytes stay in registers
+  constexpr int MAX_STEPS = 16;                  // L <= 4096 -> chunk <= 512 positions = 16 ballots per warp
+  const int chunk = ((L + nwarps * 32 - 1) / (nwarps * 32)) * 32;
+  const int c0 = wid * chunk;
+  unsigned masks[MAX_STEPS];
+  int wkept = 0;
+#pragma unroll
+  for (int it = 0; it < MAX_STEPS; ++it) {
+    const int j = c0 + it * 32 + lane;
+    const bool k = it * 32 < chunk && j < L && kp[j] != 0;
+    masks[it] = __ballot_sync(0xffffffffu, k);
+    wkept += __popc(masks[it]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+  if (lane == 0) { sh_before[wid] = before; sh_wkept[wid] = wkept; }
+  __syncthreads();
+  int out0 = 0, kept = 0, woff = 0;
+  for (int i = 0; i < nwarps; ++i) {
+    out0 += sh_before[i];
+    if (i < wid) woff += sh_wkept[i];
+    kept += sh_wkept[i];
+  }
+#pragma unroll
+  for (int it = 0; it < MAX_STEPS; ++it) {
+    const unsigned m = masks[it];
+    if ((m >> lane) & 1u) sh_pos[woff + __popc(m & ((1u << lane) - 1u))] = (unsigned short)(c0 + it * 32 + lane);
+    woff += __popc(m);
   }
   __syncthreads();
-  const int kept = sh_kept;
-  const int out0 = frame_offsets[f];
+  ET_CHECK(kept >= 0 && kept <= L && out0 >= 0 && (long long)out0 + kept <= (long long)n_cap * L, return);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    frame_offsets[f] = out0;
+    if (f == n - 1) {
+      frame_offsets[n] = out0 + kept;
+      totals[0] = n;
+      totals[1] = out0 + kept;
+    }
+  }
   for (int r = blockIdx.x * nwarps + wid; r < kept; r += gridDim.x * nwarps) {
     const int j = sh_pos[r];
+    ET_CHECK(j < L, continue);
     float4 v[NV];
     load_row<NV>(x + ((size_t)f * L + j) * D, D, lane, v);
     if (ln_g) layernorm_row_inplace<NV>(v, D, lane, ln_g, ln_b, eps);
@@ -260,16 +309,16 @@ gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restric
   }
 }
 
-void launch_gather_tokens(const float* x, const unsigned char* keep, const int* frame_offsets, int n_cap, int L, int D,
-                          const float* ln_g, const float* ln_b, float eps, float* tokens, int* token_pos,
-                          const int* n_frames_dev, cudaStream_t s) {
+void launch_gather_tokens(const float* x, const unsigned char* keep, const int* count, int* frame_offsets, int* totals,
+                          int n_cap, int L, int D, const float* ln_g, const float* ln_b, float eps, float* tokens,
+                          int* token_pos, const int* n_frames_dev, cudaStream_t s) {
   if (n_cap <= 0) return;
   const int slices = max(1, min(16, cdiv(L, 64)));
   ET_COUNT_LAUNCH();
   const int need = cdiv(D / 4, 32);      // float4 chunks per lane
 #define ET_GATHER(NV)                                                                                      \
   gather_tokens_kernel<NV><<<dim3(slices, n_cap), 256, sizeof(unsigned short) * L, s>>>(                   \
-      x, keep, frame_offsets, n_cap, L, D, ln_g, ln_b, eps, tokens, token_pos, n_frames_dev)
+      x, keep, count, frame_offsets, totals, n_cap, L, D, ln_g, ln_b, eps, tokens, token_pos, n_frames_dev)
   if (need <= 2) ET_GATHER(2);
   else if (need <= 4) ET_GATHER(4);
   else if (need <= 6) ET_GATHER(6);

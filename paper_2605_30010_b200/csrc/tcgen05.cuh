@@ -38,7 +38,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 // Bounded wait.  Returns false if the limit ran out or another role of the CTA aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   int spins = 0;
@@ -46,7 +47,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63) == 0) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; return false; }
+      if (global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
   }
 }

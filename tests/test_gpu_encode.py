@@ -182,6 +182,11 @@ def test_argument_errors(B):
     with pytest.raises(B.EarlyTomError) as ei:
         B.Encoder(wl.shape, blob[:-1], B.ET_F32, 8)
     assert ei.value.status == 7
+    poisoned = blob.copy()
+    poisoned[len(poisoned) // 2] = np.inf
+    with pytest.raises(B.EarlyTomError) as ei:
+        B.Encoder(wl.shape, poisoned, B.ET_F32, 8)
+    assert ei.value.status == 7                                      # non-finite weight
     enc = B.Encoder(wl.shape, blob, B.ET_F32, 4)
     with pytest.raises(B.EarlyTomError) as ei:
         enc.encode_batch(to_cuda(frames), offs, wl.params)          # 8 frames > capacity 4

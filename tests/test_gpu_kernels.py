@@ -68,11 +68,15 @@ def oracle_plan(sim64, offs, alpha, tau_seg, tau_merge, weighted):
             np.array(w_a), np.array(w_b), np.array(new_off))
 
 
-@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("seed", range(8))
 def test_merge_plan_matches_oracle(B, seed):
     rng = np.random.default_rng(seed)
     V = int(rng.integers(1, 6))
     lens = rng.integers(1, 40, V)
+    if seed == 6:                       # more videos than lanes, single-frame videos among them
+        V, lens = 70, rng.integers(1, 6, 70)
+    if seed == 7:                       # a list longer than the shared-memory staging area of the plan
+        V, lens = 3, np.array([1500, 1, 1700])
     offs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
     n = int(offs[-1])
     sim = rng.uniform(0.5, 1.0, n).astype(np.float32)

@@ -33,6 +33,26 @@ def test_static_scratch_matches_regular_entry_point_twice_in_a_row():
         assert torch.equal(got, want), "same kernels, same reduction order: results should be identical"
 
 
+def test_static_entry_point_takes_no_device_memory():
+    """What the entry point is for: after the first call on the device (which looks up the array's address), a call
+    neither allocates nor frees device memory -- the driver's free-byte count and torch's allocator are unchanged."""
+    import torch
+    from paper_2605_30010_b200 import binding as B
+    rng = np.random.default_rng(7)
+    x = torch.from_numpy(_video(rng, 12, 100, 64)).cuda()
+    out = torch.empty(11, dtype=torch.float32, device="cuda")
+    B.et_frame_similarity_static(x, out)                       # first call: set-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(3):
+        B.et_frame_similarity_static(x, out)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, f"device free memory changed by {free0 - free1} bytes across allocation-free calls"
+    assert torch.cuda.memory_allocated() == alloc0 and torch.cuda.memory_reserved() == reserved0
+
+
 def test_static_scratch_rejects_oversized_problems():
     import torch
     from paper_2605_30010_b200 import binding as B
