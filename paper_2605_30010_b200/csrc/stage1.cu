@@ -375,7 +375,8 @@ __global__ void __launch_bounds__(128) similarity_plan_kernel(SimPlanArgs a) {
     auto is_cross = [cross, t0](int t) { return ((cross >> (t - t0)) & 1u) != 0; };
     unsigned long long* acc = a.acc + (size_t)(l % SIM_SLOTS) * a.n_cap;
     cos_run<NV>(a.x, l, t0, t1, a.L, a.D, lane, is_cross, [=](int t, float c) {
-      if (lane == 0) atomicAdd(acc + t, (unsigned long long)__double2ll_rn((double)c * SIM_FIXED_ONE));
+      // c * 2^32 is exact in fp32 (a power-of-two scaling), so the only rounding is the one to an integer
+      if (lane == 0) atomicAdd(acc + t, (unsigned long long)__float2ll_rn(c * 4294967296.0f));
     });
   }
   if (lane == 0) __threadfence();       // this warp's additions before the block's ticket
