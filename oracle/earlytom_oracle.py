@@ -23,7 +23,8 @@ The method is a heuristic pipeline, so the oracle is the algorithm's steps in th
   cost model                 Eq. 8
 
 Pinning status (tests/test_oracle_*.py): encoder forward pinned against a composition of
-torch CPU library ops; similarity, segmentation, merge rule, weights, top-k, windows pinned by
+torch CPU library ops; similarity, segmentation, merge rule, weights (the formula and the assembled
+step, on frames whose similarities are known cosines), top-k, windows (both window modes) pinned by
 closed forms, brute force and invariants.  Readings with no external pin ("parity unpinned"):
 which tensor is compared and merged (the residual stream entering the block), the value of
 tau_merge (a parameter), the definition of the per-token attention score A (mean over heads and
@@ -429,11 +430,21 @@ def encode_video(frames: np.ndarray, shape, blob_or_w, params, dtype=np.float64,
     `forced` (tests only) replays given decisions instead of taking them:
       {"merge": {layer: (starts bool[n], merge_with_next bool[n])}, "keep": bool [N, L]}.
     """
-    w = blob_or_w if isinstance(blob_or_w, dict) else split_weights(shape, blob_or_w)
-    B = frames.shape[0]
+    arch = int(getattr(shape, "arch", 0))
+    if arch == 1:
+        # Qwen2.5-VL-style encoder (the paper's generalisation study): same method, another encoder.  A "frame" is an
+        # encoder frame (temporal_patch input frames); the encoder's pieces live in oracle/qwenvl_oracle.py.
+        from oracle import qwenvl_oracle as Q
+        w = blob_or_w if isinstance(blob_or_w, dict) else Q.split_weights(shape, blob_or_w)
+        X = Q.embed(frames.astype(dtype), shape, w)
+        block = Q.encoder_block
+    else:
+        w = blob_or_w if isinstance(blob_or_w, dict) else split_weights(shape, blob_or_w)
+        X = patchify(frames.astype(dtype), shape.patch_size) @ w["patch_w"].astype(dtype) \
+            + w["patch_b"].astype(dtype) + w["pos"].astype(dtype)[None]
+        block = encoder_block
+    B = X.shape[0]
     L, D = shape.tokens_per_frame, shape.hidden
-    X = patchify(frames.astype(dtype), shape.patch_size) @ w["patch_w"].astype(dtype) \
-        + w["patch_b"].astype(dtype) + w["pos"].astype(dtype)[None]
     meta = [FrameMeta(t, t) for t in range(B)]
     traces: List[MergeLayerTrace] = []
     A = None
@@ -449,11 +460,14 @@ def encode_video(frames: np.ndarray, shape, blob_or_w, params, dtype=np.float64,
             traces.append(tr)
         fpb.append(X.shape[0])
         last = layer == shape.num_layers - 1
-        X, sc = encoder_block(X, w, layer, shape, want_scores=last)
+        X, sc = block(X, w, layer, shape, want_scores=last)
         if last:
             A = sc
     N = X.shape[0]
-    feats = layer_norm(X, w["post_g"], w["post_b"], shape.ln_eps) if shape.post_layernorm else X
+    if arch == 1:
+        feats = Q.final_norm(X, w, shape)
+    else:
+        feats = layer_norm(X, w["post_g"], w["post_b"], shape.ln_eps) if shape.post_layernorm else X
     if not merge_layers:
         # Stage I is off: the segment list for Stage II comes from running the streaming segmentation
         # of Sec. 3.2 on the final features (Sec. 3.3 says the division follows that segmentation).
@@ -512,7 +526,13 @@ def _stage1_forced(F, meta, decision, weighted: bool, layer: int):
 def encode_batch(frames: np.ndarray, video_offsets: Sequence[int], shape, blob_or_w, params,
                  dtype=np.float64, **kw) -> List[VideoResult]:
     """Independent videos: each one goes through `encode_video` on its own."""
-    w = blob_or_w if isinstance(blob_or_w, dict) else split_weights(shape, blob_or_w)
+    if isinstance(blob_or_w, dict):
+        w = blob_or_w
+    elif int(getattr(shape, "arch", 0)) == 1:
+        from oracle import qwenvl_oracle as Q
+        w = Q.split_weights(shape, blob_or_w)
+    else:
+        w = split_weights(shape, blob_or_w)
     return [encode_video(frames[video_offsets[v]:video_offsets[v + 1]], shape, w, params, dtype=dtype, video_index=v, **kw)
             for v in range(len(video_offsets) - 1)]
 

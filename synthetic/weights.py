@@ -11,6 +11,13 @@ Blob order (all float32, row-major, a linear layer is y = x @ W + b with W [in, 
 
 wqkv's output columns are [Q | K | V], each D wide, head h at columns h*dh..(h+1)*dh of its third.
 
+Qwen2.5-VL-style encoders (shape.arch == 1) have no position table, no patch bias and no norm shifts:
+
+  patch_w [3*tp*p*p, D]   (row index = c*tp*p*p + t*p*p + dy*p + dx, tp = frames per temporal patch)
+  for each layer:  n1_g [D], wqkv [D, 3D], bqkv [3D], wo [D, D], bo [D],
+                   n2_g [D], wgu [D, 2M] (columns [gate | up]), bgu [2M], wd [M, D], bd [D]
+  post_g [D]
+
 Distributions: linear weights N(0, 1/fan_in) (attention logits come out O(1), so the
 attention scores are well separated); the two residual-branch output projections are
 additionally scaled by 1/sqrt(2*layers); biases N(0, 0.02^2); LayerNorm gains
@@ -26,6 +33,19 @@ import numpy as np
 
 def weight_layout(shape) -> List[Tuple[str, Tuple[int, ...], int]]:
     D, M, L, P = shape.hidden, shape.mlp_dim, shape.tokens_per_frame, shape.patch_dim
+    if getattr(shape, "arch", 0) == 1:
+        items = [("patch_w", (P, D))]
+        for i in range(shape.num_layers):
+            pre = f"l{i}."
+            items += [(pre + "n1_g", (D,)), (pre + "wqkv", (D, 3 * D)), (pre + "bqkv", (3 * D,)),
+                      (pre + "wo", (D, D)), (pre + "bo", (D,)), (pre + "n2_g", (D,)),
+                      (pre + "wgu", (D, 2 * M)), (pre + "bgu", (2 * M,)), (pre + "wd", (M, D)), (pre + "bd", (D,))]
+        items += [("post_g", (D,))]
+        out, off = [], 0
+        for name, shp in items:
+            out.append((name, shp, off))
+            off += int(np.prod(shp))
+        return out
     items: List[Tuple[str, Tuple[int, ...]]] = [("patch_w", (P, D)), ("patch_b", (D,)), ("pos", (L, D))]
     for i in range(shape.num_layers):
         pre = f"l{i}."
@@ -56,9 +76,9 @@ def make_weights(shape, seed: int, pos_std: float = 0.5) -> np.ndarray:
         n = int(np.prod(shp))
         leaf = name.split(".")[-1]
         z = rng.standard_normal(n, dtype=np.float32)
-        if leaf in ("patch_w", "wqkv", "wo", "w1", "w2"):
+        if leaf in ("patch_w", "wqkv", "wo", "w1", "w2", "wgu", "wd"):
             std = 1.0 / np.sqrt(shp[0])
-            if leaf in ("wo", "w2"):
+            if leaf in ("wo", "w2", "wd"):
                 std *= branch_scale
             z *= np.float32(std)
         elif leaf == "pos":
