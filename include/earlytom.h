@@ -65,8 +65,26 @@ typedef struct {
   int gelu_tanh;        /* 1 = tanh approximation of GELU, 0 = erf form */
   int post_layernorm;   /* 1 = final LayerNorm applied to the kept tokens */
   int dtype;            /* et_dtype */
-  int max_frames_total; /* capacity: sum of frames over the videos of one call, at most 65535 */
+  int max_frames_total; /* capacity: sum of (input) frames over the videos of one call; at most 65535 encoder frames */
   int max_videos;       /* capacity: videos per call */
+  /* Architecture family (zero-initialised fields give the SigLIP-style encoder described above).
+   * arch 1 = Qwen2.5-VL-style encoder, the architecture of the paper's generalisation study (supplementary
+   * "Generalizability Analysis"): RMSNorm (gain only) instead of LayerNorm, gated SiLU MLP with biases, biases on
+   * QKV / output projection, 2-D rotary positions on q and k (rotate-half pairing; the first dh/4 pairs turn with the
+   * token's row in the patch grid, the next dh/4 with its column, frequencies rope_theta^(-2i/(dh/2))), no position
+   * table, no patch-embedding bias; temporal_patch input frames form ONE encoder frame (a convolution over
+   * temporal_patch x p x p pixels); attention runs inside windows of window x window patches except in the blocks
+   * whose bit is set in full_attn_mask (bit b = 0-based block b), which attend over the whole encoder frame.
+   * Requirements for arch 1: head dim a multiple of 4; window = 0 (no windows) or a divisor of the patch grid; the
+   * last block in full_attn_mask (its attention scores feed Stage II); frame counts multiples of temporal_patch.
+   * Every frame index and count the library reports (et_result, et_trace, Eq. 5's B and N) is then in ENCODER frames.
+   * The final RMSNorm (post_layernorm) is the one that precedes the model's 2 x 2 patch merger; the merger itself is
+   * not part of this library. */
+  int arch;
+  int temporal_patch;   /* arch 1: input frames per encoder frame (>= 1); arch 0: 0 or 1 */
+  int window;           /* arch 1: window side in patches, 0 = full attention everywhere */
+  unsigned long long full_attn_mask; /* arch 1 with window > 0: blocks with full attention */
+  float rope_theta;     /* arch 1: base of the rotary frequencies, e.g. 10000 */
 } et_config;
 
 /* Host fp32 blob, row-major, y = x W + b with W [in][out], in this order:
@@ -74,6 +92,10 @@ typedef struct {
  *   per layer: ln1_g, ln1_b [D]; wqkv [D][3D] (columns Q|K|V, head h at h*dh of its third),
  *   bqkv [3D]; wo [D][D], bo [D]; ln2_g, ln2_b [D]; w1 [D][M], b1 [M]; w2 [M][D], b2 [D];
  *   then post_g, post_b [D].
+ * arch 1 (see et_config):
+ *   patch_w [3*tp*p*p][D] (row = c*tp*p*p + t*p*p + dy*p + dx),
+ *   per layer: n1_g [D]; wqkv [D][3D], bqkv [3D]; wo [D][D], bo [D]; n2_g [D]; wgu [D][2M] (columns gate | up),
+ *   bgu [2M]; wd [M][D], bd [D];   then post_g [D].
  * The library converts and copies; the caller may free the blob after create returns. */
 typedef struct {
   const float* data;

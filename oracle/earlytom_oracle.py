@@ -50,6 +50,9 @@ WSUM_EPS = 1e-6     # Eq. 3 denominator guard: below it the merge is a plain mea
 
 def split_weights(shape, blob: np.ndarray) -> Dict[str, np.ndarray]:
     """Views into the fp32 blob in the library's documented order (see include/earlytom.h)."""
+    if int(getattr(shape, "arch", 0)) == 1:
+        from oracle import qwenvl_oracle as Q
+        return Q.split_weights(shape, blob)
     D, M, L = shape.hidden, shape.mlp_dim, shape.tokens_per_frame
     P = 3 * shape.patch_size * shape.patch_size
     out: Dict[str, np.ndarray] = {}

@@ -41,7 +41,9 @@ class EarlyTomError(RuntimeError):
 class et_config(C.Structure):
     _fields_ = [("image_size", C.c_int), ("patch_size", C.c_int), ("num_layers", C.c_int), ("hidden", C.c_int),
                 ("heads", C.c_int), ("mlp_dim", C.c_int), ("ln_eps", C.c_float), ("gelu_tanh", C.c_int),
-                ("post_layernorm", C.c_int), ("dtype", C.c_int), ("max_frames_total", C.c_int), ("max_videos", C.c_int)]
+                ("post_layernorm", C.c_int), ("dtype", C.c_int), ("max_frames_total", C.c_int), ("max_videos", C.c_int),
+                ("arch", C.c_int), ("temporal_patch", C.c_int), ("window", C.c_int), ("full_attn_mask", C.c_ulonglong),
+                ("rope_theta", C.c_float)]
 
 
 class et_weights(C.Structure):
@@ -341,7 +343,9 @@ class Encoder:
     def __init__(self, shape, weights: np.ndarray, dtype: int, max_frames_total: int, max_videos: int = 1):
         cfg = et_config(shape.image_size, shape.patch_size, shape.num_layers, shape.hidden, shape.heads, shape.mlp_dim,
                         float(shape.ln_eps), int(shape.gelu_tanh), int(shape.post_layernorm), int(dtype),
-                        int(max_frames_total), int(max_videos))
+                        int(max_frames_total), int(max_videos), int(getattr(shape, "arch", 0)),
+                        int(getattr(shape, "temporal_patch", 1)), int(getattr(shape, "window", 0)),
+                        int(getattr(shape, "full_attn_mask", 0)), float(getattr(shape, "rope_theta", 0.0)))
         self.handle = et_encoder_create(cfg, weights)
         self.num_layers = shape.num_layers
         self.shape = shape

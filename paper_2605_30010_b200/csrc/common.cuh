@@ -82,9 +82,18 @@ enum Epilogue : int { EPI_STORE = 0, EPI_GELU = 1, EPI_RESIDUAL = 2, EPI_TABLE =
 
 // ---- elementwise.cu ------------------------------------------------------------------------
 // frames fp32 [T][3][H][W] -> patches [T*L][k_pad] (zero padded beyond 3*p*p), fp32 or bf16.
+// tp input frames make one encoder frame (T counts encoder frames); int2raster: optional internal token order.
 void launch_im2col(const float* frames, void* patches, int T, int image, int patch, int k_pad, bool out_bf16,
-                   const int* n_frames_dev, cudaStream_t s);
-// LayerNorm of rows [rows_cap][D]; live rows = *n_frames_dev * rows_per_frame when n_frames_dev != NULL.
+                   const int* n_frames_dev, cudaStream_t s, int tp = 1, const int* int2raster = nullptr);
+// 2-D rotary positions in place on the Q and K parts of packed rows [rows][3*heads*dh]; table [L][dh/2] (cos, sin)
+void launch_rope_pairs(void* qkv, const float2* table, int rows_cap, int L, int heads, int dh, bool is_bf16,
+                       const int* n_frames_dev, cudaStream_t s);
+// h[r][j] = silu(gu[r][j]) * gu[r][Mp + j], j < Mp
+void launch_gated_silu(const void* gu, void* h, int rows_cap, int Mp, bool is_bf16, const int* n_frames_dev,
+                       int rows_per_frame, cudaStream_t s);
+void launch_scale_count(const int* in, int mult, int* out, cudaStream_t s);
+// LayerNorm of rows [rows_cap][D] (RMSNorm with gain g when b == NULL); live rows = *n_frames_dev * rows_per_frame
+// when n_frames_dev != NULL.
 void launch_layernorm(const float* x, const float* g, const float* b, float eps, void* y, int rows_cap, int D,
                       bool out_bf16, const int* n_frames_dev, int rows_per_frame, cudaStream_t s);
 
@@ -210,6 +219,7 @@ struct SelectArgs {
   const int* orig_vid_off;   // [V+1] offsets of the input videos (for B of Eq. 5)
   int n_cap, n_videos, L, selection, retain_mode, window_mode;
   int mask_given;            // 1: keep[] was provided by the caller; write only the flags and amounts
+  const int* raster2int;     // NULL, or the internal position of raster position j (scores are in internal order)
   double retain;
   unsigned char* dynamic;    // [Fmax] out
   unsigned char* keep;       // [Fmax][L] out
@@ -234,6 +244,8 @@ void launch_scan_counts(const int* count, int* frame_offsets, int* totals, int n
 // totals[1] = n_tokens
 void launch_gather_tokens(const float* x, const unsigned char* keep, const int* count, int* frame_offsets, int* totals,
                           int n_cap, int L, int D, const float* ln_g, const float* ln_b, float eps, float* tokens,
-                          int* token_pos, const int* n_frames_dev, cudaStream_t s);
+                          int* token_pos, const int* n_frames_dev, cudaStream_t s, const int* raster2int = nullptr);
+// (ln_b == NULL with ln_g != NULL: RMSNorm with gain ln_g; raster2int: the keep mask and token_pos are in raster
+// order while the rows of x are in the encoder's internal order)
 
 }  // namespace et

@@ -12,27 +12,34 @@ namespace et {
 __device__ __forceinline__ void store_pair(float* p, float a, float b) { *reinterpret_cast<float2*>(p) = make_float2(a, b); }
 __device__ __forceinline__ void store_pair(bf16* p, float a, float b) { *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b); }
 
+// `tp` input frames form one encoder frame (temporal patch): feature index = ((c*tp + t)*p + dy)*p + dx, the
+// flattening of a [D][3][tp][p][p] convolution weight.  With `int2raster` the tokens of an encoder frame are written
+// in the encoder's internal order (token l of the output sits at raster position int2raster[l] of the patch grid).
 template <typename T>
 __global__ void im2col_kernel(const float* __restrict__ frames, T* __restrict__ patches, int T_frames, int image,
-                              int patch, int grid, int k_pad, const int* __restrict__ n_frames_dev) {
-  const int n_frames = n_frames_dev ? min(*n_frames_dev, T_frames) : T_frames;
+                              int patch, int grid, int k_pad, int tp, const int* __restrict__ int2raster,
+                              const int* __restrict__ n_frames_dev) {
+  const int n_frames = n_frames_dev ? min(*n_frames_dev, T_frames) : T_frames;      // encoder frames
   const int L = grid * grid;
-  const int rows_per_tok = 3 * patch + 1;  // 3*p pixel rows + one job that writes the zero pad
+  const int rows_per_tok = 3 * tp * patch + 1;  // 3*tp*p pixel rows + one job that writes the zero pad
   const long long total = (long long)n_frames * L * rows_per_tok;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int job = (int)(idx % rows_per_tok);
     const long long tok = idx / rows_per_tok;
     T* dst_row = patches + tok * k_pad;
-    if (job == 3 * patch) {
-      for (int c = 3 * patch * patch; c < k_pad; ++c) dst_row[c] = to_out<T>(0.f);
+    if (job == 3 * tp * patch) {
+      for (int c = 3 * tp * patch * patch; c < k_pad; ++c) dst_row[c] = to_out<T>(0.f);
       continue;
     }
-    const int c = job / patch, dy = job % patch;
-    const int f = (int)(tok / L), l = (int)(tok % L);
+    const int ct = job / patch, dy = job % patch;       // ct = c*tp + t
+    const int c = ct / tp, t = ct % tp;
+    const int f = (int)(tok / L);
+    int l = (int)(tok % L);
+    if (int2raster) l = int2raster[l];
     const int gy = l / grid, gx = l % grid;
-    const float* src = frames + (((long long)f * 3 + c) * image + (gy * patch + dy)) * image + gx * patch;
-    T* dst = dst_row + (c * patch + dy) * patch;
+    const float* src = frames + ((((long long)f * tp + t) * 3 + c) * image + (gy * patch + dy)) * image + gx * patch;
+    T* dst = dst_row + (ct * patch + dy) * patch;
     if ((patch & 1) == 0 && (image & 1) == 0 && (k_pad & 1) == 0 && (reinterpret_cast<size_t>(frames) & 7) == 0) {
       // pixel pairs: the patch row starts at an even pixel of an even-width image and at an even patch column
       const float2* s2 = reinterpret_cast<const float2*>(src);
@@ -47,23 +54,23 @@ __global__ void im2col_kernel(const float* __restrict__ frames, T* __restrict__ 
 }
 
 void launch_im2col(const float* frames, void* patches, int T, int image, int patch, int k_pad, bool out_bf16,
-                   const int* n_frames_dev, cudaStream_t s) {
+                   const int* n_frames_dev, cudaStream_t s, int tp, const int* int2raster) {
   const int grid = image / patch;
-  const long long total = (long long)T * grid * grid * (3 * patch + 1);
+  const long long total = (long long)T * grid * grid * (3 * tp * patch + 1);
   const int threads = 256;
   long long want = (total + threads - 1) / threads;
   const int blocks = (int)(want < 148LL * 32 ? want : 148LL * 32);
   if (blocks == 0) return;
   ET_COUNT_LAUNCH();
   if (out_bf16)
-    im2col_kernel<bf16><<<blocks, threads, 0, s>>>(frames, (bf16*)patches, T, image, patch, grid, k_pad, n_frames_dev);
+    im2col_kernel<bf16><<<blocks, threads, 0, s>>>(frames, (bf16*)patches, T, image, patch, grid, k_pad, tp, int2raster, n_frames_dev);
   else
-    im2col_kernel<float><<<blocks, threads, 0, s>>>(frames, (float*)patches, T, image, patch, grid, k_pad, n_frames_dev);
+    im2col_kernel<float><<<blocks, threads, 0, s>>>(frames, (float*)patches, T, image, patch, grid, k_pad, tp, int2raster, n_frames_dev);
 }
 
 // ---------------------------------------------------------------------------------------------
 // LayerNorm: one warp per row, row held in registers, mean then centred variance (two passes over
-// registers), fp32 statistics.
+// registers), fp32 statistics.  With b == NULL the kernel computes RMSNorm, y = x / sqrt(mean(x^2) + eps) * g.
 // ---------------------------------------------------------------------------------------------
 template <typename T, int NV>
 __global__ void __launch_bounds__(256)
@@ -75,7 +82,8 @@ layernorm_kernel(const float* __restrict__ x, const float* __restrict__ g, const
   for (int row = blockIdx.x * warps_per_block + (threadIdx.x >> 5); row < rows; row += gridDim.x * warps_per_block) {
     float4 v[NV];
     load_row<NV>(x + (size_t)row * D, D, lane, v);
-    layernorm_row_inplace<NV>(v, D, lane, g, b, eps);
+    if (b) layernorm_row_inplace<NV>(v, D, lane, g, b, eps);
+    else rmsnorm_row_inplace<NV>(v, D, lane, g, eps);          // no shift given: RMSNorm with gain g
     store_row<NV>(y + (size_t)row * D, D, lane, v);
   }
 }
@@ -103,6 +111,77 @@ void launch_layernorm(const float* x, const float* g, const float* b, float eps,
   ET_COUNT_LAUNCH();
   if (out_bf16) launch_layernorm_t<bf16>(x, g, b, eps, (bf16*)y, rows_cap, D, n_frames_dev, rows_per_frame, s);
   else launch_layernorm_t<float>(x, g, b, eps, (float*)y, rows_cap, D, n_frames_dev, rows_per_frame, s);
+}
+
+// ---------------------------------------------------------------------------------------------
+// 2-D rotary positions on the Q and K parts of packed rows [rows][3*D] (Q | K | V, head h at h*dh of its third):
+// pair (x[i], x[i + dh/2]) of every head is turned by the angle of (token position in its frame, i); table
+// [L][dh/2] holds (cos, sin).  One thread per (row, head, pair) for Q and K alike.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void rope_pairs_kernel(T* __restrict__ qkv, const float2* __restrict__ table, int rows_cap, int L, int heads,
+                                  int dh, const int* __restrict__ n_frames_dev) {
+  const int rows = n_frames_dev ? min(rows_cap, *n_frames_dev * L) : rows_cap;
+  const int half = dh >> 1, D = heads * dh;
+  const long long per_row = 2LL * heads * half;
+  const long long total = (long long)rows * per_row;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(idx / per_row);
+    int rem = (int)(idx % per_row);
+    const int which = rem / (heads * half);             // 0 = Q, 1 = K
+    rem %= heads * half;
+    const int h = rem / half, i = rem % half;
+    const float2 cs = __ldg(table + (size_t)(r % L) * half + i);
+    T* p = qkv + (size_t)r * 3 * D + (size_t)which * D + h * dh + i;
+    const float a = (float)p[0], b = (float)p[half];
+    p[0] = to_out<T>(a * cs.x - b * cs.y);
+    p[half] = to_out<T>(b * cs.x + a * cs.y);
+  }
+}
+
+void launch_rope_pairs(void* qkv, const float2* table, int rows_cap, int L, int heads, int dh, bool is_bf16,
+                       const int* n_frames_dev, cudaStream_t s) {
+  if (rows_cap <= 0) return;
+  const long long total = (long long)rows_cap * heads * dh;
+  const int blocks = (int)min((total + 255) / 256, 148LL * 32);
+  ET_COUNT_LAUNCH();
+  if (is_bf16) rope_pairs_kernel<bf16><<<blocks, 256, 0, s>>>((bf16*)qkv, table, rows_cap, L, heads, dh, n_frames_dev);
+  else rope_pairs_kernel<float><<<blocks, 256, 0, s>>>((float*)qkv, table, rows_cap, L, heads, dh, n_frames_dev);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Gated activation: h[r][j] = silu(gu[r][j]) * gu[r][Mp + j] for j < Mp (gu has 2*Mp columns: gate | up).
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void gated_silu_kernel(const T* __restrict__ gu, T* __restrict__ h, int rows_cap, int Mp,
+                                  const int* __restrict__ n_frames_dev, int rows_per_frame) {
+  const int rows = n_frames_dev ? min(rows_cap, *n_frames_dev * rows_per_frame) : rows_cap;
+  const long long total = (long long)rows * Mp;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const long long r = idx / Mp;
+    const int j = (int)(idx % Mp);
+    const float g = (float)gu[r * 2 * Mp + j], u = (float)gu[r * 2 * Mp + Mp + j];
+    h[idx] = to_out<T>(g / (1.f + expf(-g)) * u);
+  }
+}
+
+void launch_gated_silu(const void* gu, void* h, int rows_cap, int Mp, bool is_bf16, const int* n_frames_dev,
+                       int rows_per_frame, cudaStream_t s) {
+  if (rows_cap <= 0) return;
+  const long long total = (long long)rows_cap * Mp;
+  const int blocks = (int)min((total + 255) / 256, 148LL * 32);
+  ET_COUNT_LAUNCH();
+  if (is_bf16) gated_silu_kernel<bf16><<<blocks, 256, 0, s>>>((const bf16*)gu, (bf16*)h, rows_cap, Mp, n_frames_dev, rows_per_frame);
+  else gated_silu_kernel<float><<<blocks, 256, 0, s>>>((const float*)gu, (float*)h, rows_cap, Mp, n_frames_dev, rows_per_frame);
+}
+
+// out[0] = in[0] * mult (the number of attention windows alive = frames alive * windows per frame)
+__global__ void scale_count_kernel(const int* __restrict__ in, int mult, int* __restrict__ out) { out[0] = in[0] * mult; }
+void launch_scale_count(const int* in, int mult, int* out, cudaStream_t s) {
+  ET_COUNT_LAUNCH();
+  scale_count_kernel<<<1, 1, 0, s>>>(in, mult, out);
 }
 
 }  // namespace et

@@ -19,8 +19,10 @@ void launch_score_finish(const float* partial, float* score, int n_cap, int L, i
 
 namespace {
 
-// dst[n][k_pad] (bf16, zero padded for k >= K) = src[k][n] (fp32)
-__global__ void transpose_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int K, int N, int k_pad) {
+// dst[row(n)][k_pad] (bf16, zero padded for k >= K) = src[k][n] (fp32); row(n) = n for n < split, n + shift beyond
+// (the [gate | up] weight of a gated MLP is stored with each half padded to the same width)
+__global__ void transpose_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int K, int N, int k_pad,
+                                         int split, int shift) {
   __shared__ float tile[32][33];
   const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
   for (int i = threadIdx.y; i < 32; i += blockDim.y) {
@@ -30,7 +32,7 @@ __global__ void transpose_to_bf16_kernel(const float* __restrict__ src, bf16* __
   __syncthreads();
   for (int i = threadIdx.y; i < 32; i += blockDim.y) {
     const int n = n0 + i, k = k0 + threadIdx.x;
-    if (n < N && k < k_pad) dst[(size_t)n * k_pad + k] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+    if (n < N && k < k_pad) dst[(size_t)(n < split ? n : n + shift) * k_pad + k] = __float2bfloat16_rn(tile[threadIdx.x][i]);
   }
 }
 
@@ -45,7 +47,7 @@ __global__ void find_nonfinite_kernel(const float* __restrict__ w, size_t count,
 struct LayerOffsets { size_t ln1_g, ln1_b, wqkv, bqkv, wo, bo, ln2_g, ln2_b, w1, b1, w2, b2; };
 
 struct LayerBf16 {
-  bf16 *wqkv_t, *wo_t, *w1_t, *w2_t;
+  bf16 *wqkv_t, *wo_t, *w1_t, *w2_t;       // arch 1: w1 = [gate | up] (each half padded to Mp rows), w2 = down
   WeightDesc d_wqkv, d_wo, d_w1, d_w2;
 };
 
@@ -56,8 +58,20 @@ using namespace et;
 
 struct et_encoder {
   et_config cfg{};
-  int L = 0, grid = 0, P = 0, Kp = 0, dh = 0, Fmax = 0, Vmax = 0;
+  int L = 0, grid = 0, P = 0, Kp = 0, dh = 0, Fmax = 0, Vmax = 0;   // Fmax: capacity in ENCODER frames
   bool bf = false;
+  // Qwen2.5-VL-style encoder (cfg.arch == 1)
+  int arch = 0, tp = 1, ws = 0, wpf = 1, Lw = 0, Mp = 0;   // frames per temporal patch, window side, windows per frame,
+                                                            // tokens per window, MLP width as stored (padded on the bf16 path)
+  int *int2raster = nullptr, *raster2int = nullptr;         // [L] token orders (NULL: raster order is the internal order)
+  std::vector<int> r2i_host;                                // host copy of raster2int (the trace reports scores in raster order)
+  float* h_scores_int = nullptr;                            // staging for that permutation
+  float2* rope_table = nullptr;                             // [L][dh/2] (cos, sin) by internal position
+  float* zeros = nullptr;                                   // [max(D, 2*Mp)] zero bias / zero position row
+  float* bgu_pad = nullptr;                                 // [layers][2*Mp] gate | up biases in the padded layout (bf16 path)
+  int* n_windows = nullptr;                                 // [1] attention windows alive = frames alive * wpf
+  void* GU = nullptr;                                       // [rows][2*Mp] gate | up pre-activations
+  TmaDesc c_GU;
   int device = 0;
   std::string last_error;
   std::vector<void*> dev_allocs, host_allocs;
@@ -182,6 +196,10 @@ et_status halloc(et_encoder* e, T** p, size_t count) {
 
 size_t blob_floats(const et_config& c, int L, int P) {
   const size_t D = c.hidden, M = c.mlp_dim;
+  if (c.arch == 1) {
+    const size_t per_layer = D + D * 3 * D + 3 * D + D * D + D + D + D * 2 * M + 2 * M + M * D + D;
+    return (size_t)P * D + per_layer * c.num_layers + D;
+  }
   size_t per_layer = 2 * D + D * 3 * D + 3 * D + D * D + D + 2 * D + D * M + M + M * D + D;
   return (size_t)P * D + D + (size_t)L * D + per_layer * c.num_layers + 2 * D;
 }
@@ -197,10 +215,24 @@ et_status validate_config(const et_config* c) {
   if (c->dtype != ET_F32 && c->dtype != ET_BF16) return ET_ERR_INVALID_ARG;
   if (c->dtype == ET_BF16 && (c->hidden % 8 != 0 || c->mlp_dim % 8 != 0 || (c->hidden / c->heads) % 8 != 0)) return ET_ERR_SHAPE;
   if (c->max_frames_total < 1 || c->max_videos < 1 || c->max_videos > 1024) return ET_ERR_INVALID_ARG;
-  if (c->max_frames_total > 65535) return ET_ERR_CAPACITY;      // frames index gridDim.y of the merge and gather kernels
+  if (c->max_frames_total / (c->temporal_patch > 1 ? c->temporal_patch : 1) > 65535) return ET_ERR_CAPACITY;   // frames index gridDim.y
+  if (c->arch == 1 && c->temporal_patch >= 1 && c->max_frames_total < c->temporal_patch) return ET_ERR_INVALID_ARG;
   const long long L = (long long)(c->image_size / c->patch_size) * (c->image_size / c->patch_size);
   if (L > 4096 || L * c->max_frames_total > (1ll << 30)) return ET_ERR_CAPACITY;
   if (!(c->ln_eps > 0.f)) return ET_ERR_INVALID_ARG;
+  if (c->arch == 0) {
+    if (c->temporal_patch > 1 || c->window != 0) return ET_ERR_INVALID_ARG;
+  } else if (c->arch == 1) {
+    const int g = c->image_size / c->patch_size, dh = c->hidden / c->heads;
+    if (c->temporal_patch < 1 || c->temporal_patch > 8 || c->window < 0) return ET_ERR_INVALID_ARG;
+    if (dh % 4 != 0 || !(c->rope_theta > 1.f)) return ET_ERR_SHAPE;
+    if (c->window > 0) {
+      if (g % c->window != 0) return ET_ERR_SHAPE;                                  // whole windows only
+      if (!((c->full_attn_mask >> (c->num_layers - 1)) & 1ull)) return ET_ERR_SHAPE; // Stage II needs whole-frame scores
+    }
+  } else {
+    return ET_ERR_INVALID_ARG;
+  }
   return ET_OK;
 }
 
@@ -249,9 +281,12 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
   ET_TRY(validate_params(e, p) == ET_OK ? ET_OK : fail(e, ET_ERR_INVALID_ARG, "invalid et_params"));
   if (V < 1 || V > e->Vmax) return fail(e, ET_ERR_CAPACITY, "number of videos outside [1, max_videos]");
   if (vid_off_host[0] != 0) return fail(e, ET_ERR_INVALID_ARG, "video_offsets[0] must be 0");
-  for (int v = 0; v < V; ++v)
+  for (int v = 0; v < V; ++v) {
     if (vid_off_host[v + 1] <= vid_off_host[v]) return fail(e, ET_ERR_INVALID_ARG, "every video needs at least one frame");
-  const int T = vid_off_host[V];
+    if (vid_off_host[v + 1] % e->tp != 0) return fail(e, ET_ERR_INVALID_ARG, "frame counts must be multiples of temporal_patch");
+  }
+  // From here on a frame is an ENCODER frame (temporal_patch input frames; the same thing when temporal_patch is 1).
+  const int T = vid_off_host[V] / e->tp;
   if (T > e->Fmax) return fail(e, ET_ERR_CAPACITY, "more frames than max_frames_total");
   const et_forced_plan* fp = p->forced_plan;
   if (fp) {
@@ -271,7 +306,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
   const int rows_cap = T * L;
   const float* W = e->w_blob;
 
-  memcpy(e->h_vid_off, vid_off_host, sizeof(int) * (V + 1));
+  for (int v = 0; v <= V; ++v) e->h_vid_off[v] = vid_off_host[v] / e->tp;
   ET_CUDA(e, cudaMemcpyAsync(e->orig_vid_off, e->h_vid_off, sizeof(int) * (V + 1), cudaMemcpyHostToDevice, s));
   ET_CUDA(e, cudaMemsetAsync(e->d_small, 0, sizeof(int) * 16, s));
   if (fp) {
@@ -290,9 +325,11 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
   launch_init_frames(e->fl[0], e->orig_vid_off, V, T, s);
 
   // patch embedding: im2col + dense layer with the position table added in the epilogue
-  PROF(ET_CAT_IM2COL, launch_im2col(frames_dev, e->Pm, T, c.image_size, c.patch_size, e->Kp, e->bf, nullptr, s));
-  PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Pm, e->d_Pm, W + e->off_patch_w, e->d_patch_w, e->c_X[cur], W + e->off_patch_b, e->X[cur], rows_cap, D,
-               e->bf ? e->Kp : e->P, EPI_TABLE, W + e->off_pos, L, nullptr, s)));
+  const bool qw = e->arch == 1;           // Qwen2.5-VL-style blocks
+  PROF(ET_CAT_IM2COL, launch_im2col(frames_dev, e->Pm, T, c.image_size, c.patch_size, e->Kp, e->bf, nullptr, s, e->tp, e->int2raster));
+  PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Pm, e->d_Pm, W + e->off_patch_w, e->d_patch_w, e->c_X[cur], qw ? e->zeros : W + e->off_patch_b, e->X[cur], rows_cap, D,
+               e->bf ? e->Kp : e->P, EPI_TABLE, qw ? e->zeros : W + e->off_pos, qw ? 1 : L, nullptr, s)));
+  if (e->ws > 0) launch_scale_count(e->fl[0].n, e->wpf, e->n_windows, s);
 
   int mi = 0;
   for (int layer = 0; layer < c.num_layers; ++layer) {
@@ -308,19 +345,25 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
       a.n_hist_slot = e->d_small + 2 + mi; a.status = e->d_small + 10;
       PROF(ET_CAT_SIMILARITY, launch_similarity_plan(sim_plan_args(e, e->X[cur], T, lst, V, a), s));
       PROF(ET_CAT_MERGE, launch_merge_frames(e->X[cur], e->X[cur ^ 1], T, L * D, e->fl[lst ^ 1].n, e->plan, s));
+      if (e->ws > 0) launch_scale_count(e->fl[lst ^ 1].n, e->wpf, e->n_windows, s);
       cur ^= 1; lst ^= 1; ++mi;
     }
     const int* n_dev = e->fl[lst].n;
     const LayerOffsets& o = e->lo[layer];
     const LayerBf16* b = e->bf ? &e->lb[layer] : nullptr;
     static const WeightDesc none{};
-    PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln1_g, W + o.ln1_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
+    PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln1_g, qw ? nullptr : W + o.ln1_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
     PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.wqkv, b ? b->d_wqkv : none, e->c_QKV, W + o.bqkv, e->QKV, rows_cap, 3 * D, D, EPI_STORE,
                  nullptr, 1, n_dev, s)));
+    if (qw) PROF(ET_CAT_ATTENTION, launch_rope_pairs(e->QKV, e->rope_table, rows_cap, L, H, dh, e->bf, n_dev, s));
+    // attention items: whole frames, or (in a window block) the windows, which are runs of Lw rows in the internal order
+    const bool windowed = e->ws > 0 && !((c.full_attn_mask >> layer) & 1ull);
+    const int a_cap = windowed ? T * e->wpf : T, a_L = windowed ? e->Lw : L;
+    const int* a_n = windowed ? e->n_windows : n_dev;
     PROF(ET_CAT_ATTENTION, {
-      if (e->attn_tc) ET_CUDA(e, launch_attention_tc(e->attn_maps, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, e->d_small + 10, s));
-      else if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, s);
-      else launch_attention_f32((const float*)e->QKV, (float*)e->O, e->lse, T, L, H, dh, n_dev, s);
+      if (e->attn_tc) ET_CUDA(e, launch_attention_tc(e->attn_maps, (bf16*)e->O, e->lse, a_cap, a_L, H, dh, a_n, e->d_small + 10, s));
+      else if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, a_cap, a_L, H, dh, a_n, s);
+      else launch_attention_f32((const float*)e->QKV, (float*)e->O, e->lse, a_cap, a_L, H, dh, a_n, s);
     });
     if (layer == c.num_layers - 1) {
       PROF(ET_CAT_SCORES, {
@@ -331,11 +374,21 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     }
     PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->O, e->d_O, W + o.wo, b ? b->d_wo : none, e->c_X[cur], W + o.bo, e->X[cur], rows_cap, D, D, EPI_RESIDUAL,
                  nullptr, 1, n_dev, s)));
-    PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln2_g, W + o.ln2_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
-    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, e->c_Hm, W + o.b1, e->Hm, rows_cap, Mlp, D, EPI_GELU, nullptr, 1,
-                 n_dev, s)));
-    PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, e->c_X[cur], W + o.b2, e->X[cur], rows_cap, D, Mlp, EPI_RESIDUAL,
-                 nullptr, 1, n_dev, s)));
+    PROF(ET_CAT_LAYERNORM, launch_layernorm(e->X[cur], W + o.ln2_g, qw ? nullptr : W + o.ln2_b, c.ln_eps, e->Xn, rows_cap, D, e->bf, n_dev, L, s));
+    if (qw) {
+      // gated MLP: [gate | up] pre-activations, silu(gate) * up, down projection added to the residual stream
+      const int Mp = e->Mp;
+      PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, e->c_GU, e->bf ? e->bgu_pad + (size_t)layer * 2 * Mp : W + o.b1,
+                   e->GU, rows_cap, 2 * Mp, D, EPI_STORE, nullptr, 1, n_dev, s)));
+      PROF(ET_CAT_GEMM, launch_gated_silu(e->GU, e->Hm, rows_cap, Mp, e->bf, n_dev, L, s));
+      PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, e->c_X[cur], W + o.b2, e->X[cur], rows_cap, D, Mp, EPI_RESIDUAL,
+                   nullptr, 1, n_dev, s)));
+    } else {
+      PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, e->c_Hm, W + o.b1, e->Hm, rows_cap, Mlp, D, EPI_GELU, nullptr, 1,
+                   n_dev, s)));
+      PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, e->c_X[cur], W + o.b2, e->X[cur], rows_cap, D, Mlp, EPI_RESIDUAL,
+                   nullptr, 1, n_dev, s)));
+    }
   }
   const int* n_dev = e->fl[lst].n;
   if (p->num_merge_layers == 0) {
@@ -351,6 +404,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
   sa.scores = e->scores; sa.fl = e->fl[lst]; sa.orig_vid_off = e->orig_vid_off; sa.n_cap = T; sa.n_videos = V; sa.L = L;
   sa.selection = p->selection; sa.retain_mode = p->retain_mode; sa.window_mode = p->window_mode; sa.retain = p->retain;
   sa.dynamic = e->dynamic; sa.keep = e->keep; sa.count = e->count; sa.video_k = e->video_k; sa.video_w = e->video_w;
+  sa.raster2int = e->raster2int;
   if (fp && fp->keep) {
     memcpy(e->h_keep_stage, fp->keep, (size_t)fp->n_final * L);
     ET_CUDA(e, cudaMemcpyAsync(e->keep, e->h_keep_stage, (size_t)fp->n_final * L, cudaMemcpyHostToDevice, s));
@@ -365,8 +419,8 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     PROF(ET_CAT_SELECT, launch_select_video_tokens(sa, s));
   }
   PROF(ET_CAT_GATHER, launch_gather_tokens(e->X[cur], e->keep, e->count, e->frame_offsets, e->d_small, T, L, D,
-                       c.post_layernorm ? W + e->off_post_g : nullptr, c.post_layernorm ? W + e->off_post_b : nullptr,
-                       c.ln_eps, e->tokens, e->token_pos, n_dev, s));
+                       c.post_layernorm ? W + e->off_post_g : nullptr, (c.post_layernorm && !qw) ? W + e->off_post_b : nullptr,
+                       c.ln_eps, e->tokens, e->token_pos, n_dev, s, e->raster2int));
   ET_CUDA(e, cudaMemcpyAsync(e->h_small, e->d_small, sizeof(int) * 16, cudaMemcpyDeviceToHost, s));
   ET_CUDA(e, cudaGetLastError());
   ET_CUDA(e, cudaStreamSynchronize(s));
@@ -399,7 +453,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     // algorithmic work of this call from the frame counts it actually ran with
     const double dL = L, dD = D, dM = Mlp, es = e->bf ? 2.0 : 4.0;
     double* wk = e->prof.work;
-    wk[ET_CAT_IM2COL] += (double)T * 3.0 * c.image_size * c.image_size * 4.0 + (double)T * dL * e->Kp * es;
+    wk[ET_CAT_IM2COL] += (double)T * e->tp * 3.0 * c.image_size * c.image_size * 4.0 + (double)T * dL * e->Kp * es;
     wk[ET_CAT_GEMM] += 2.0 * T * dL * dD * e->P;
     int n_in = T;
     for (int layer = 0, m = 0; layer < c.num_layers; ++layer) {
@@ -410,8 +464,9 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
         n_in = n_out; ++m;
       }
       const double rows = (double)r.frames_per_block[layer] * dL;
-      wk[ET_CAT_GEMM] += 2.0 * rows * (4.0 * dD * dD + 2.0 * dD * dM);
-      wk[ET_CAT_ATTENTION] += 4.0 * rows * dL * dD;
+      const bool windowed = e->ws > 0 && !((c.full_attn_mask >> layer) & 1ull);
+      wk[ET_CAT_GEMM] += 2.0 * rows * (4.0 * dD * dD + (qw ? 3.0 : 2.0) * dD * dM);
+      wk[ET_CAT_ATTENTION] += 4.0 * rows * (windowed ? (double)e->Lw : dL) * dD;
       wk[ET_CAT_LAYERNORM] += 2.0 * rows * dD * (4.0 + es);
     }
     if (p->num_merge_layers == 0) wk[ET_CAT_SIMILARITY] += (double)N * dL * dD * 4.0;
@@ -438,11 +493,15 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
       t.sim[i] = hs; t.ema[i] = he; t.seg_start[i] = hb; t.merge_next[i] = hm;
       n_in = t.n_out[i];
     }
-    ET_CUDA(e, cudaMemcpyAsync(e->h_scores, e->scores, sizeof(float) * (size_t)N * L, cudaMemcpyDeviceToHost, s));
+    ET_CUDA(e, cudaMemcpyAsync(e->raster2int ? e->h_scores_int : e->h_scores, e->scores, sizeof(float) * (size_t)N * L, cudaMemcpyDeviceToHost, s));
     ET_CUDA(e, cudaMemcpyAsync(e->h_keep, e->keep, (size_t)N * L, cudaMemcpyDeviceToHost, s));
     ET_CUDA(e, cudaMemcpyAsync(e->h_video_kw, e->video_k, sizeof(int) * V, cudaMemcpyDeviceToHost, s));
     ET_CUDA(e, cudaMemcpyAsync(e->h_video_kw + e->Vmax, e->video_w, sizeof(int) * V, cudaMemcpyDeviceToHost, s));
     ET_CUDA(e, cudaStreamSynchronize(s));
+    if (e->raster2int) {                // the device holds the scores in the internal token order; the trace is in raster order
+      for (int f = 0; f < N; ++f)
+        for (int j = 0; j < L; ++j) e->h_scores[(size_t)f * L + j] = e->h_scores_int[(size_t)f * L + e->r2i_host[j]];
+    }
     t.scores = e->h_scores; t.keep = e->h_keep; t.video_k = e->h_video_kw; t.video_w = e->h_video_kw + e->Vmax;
     r.trace = &t;
   }
@@ -461,7 +520,8 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return ET_ERR_CUDA;
   const int g = config->image_size / config->patch_size;
-  const int L = g * g, P = 3 * config->patch_size * config->patch_size;
+  const int tp = config->arch == 1 ? config->temporal_patch : 1;
+  const int L = g * g, P = 3 * tp * config->patch_size * config->patch_size;
   if (weights->count != blob_floats(*config, L, P)) return ET_ERR_WEIGHTS;
 
   et_encoder* e = new (std::nothrow) et_encoder();
@@ -471,22 +531,38 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   e->L = L; e->grid = g; e->P = P; e->dh = config->hidden / config->heads;
   e->bf = config->dtype == ET_BF16;
   e->Kp = e->bf ? (P + 7) / 8 * 8 : P;
-  e->Fmax = config->max_frames_total; e->Vmax = config->max_videos;
+  e->arch = config->arch; e->tp = tp;
+  e->ws = config->arch == 1 ? config->window : 0;
+  e->wpf = e->ws > 0 ? (g / e->ws) * (g / e->ws) : 1;
+  e->Lw = e->ws > 0 ? e->ws * e->ws : L;
+  e->Mp = (config->arch == 1 && e->bf) ? (config->mlp_dim + 63) / 64 * 64 : config->mlp_dim;
+  e->Fmax = config->max_frames_total / tp; e->Vmax = config->max_videos;
   if (cudaGetDevice(&e->device) != cudaSuccess) return bail(ET_ERR_CUDA);
   const size_t D = config->hidden, M = config->mlp_dim, F = e->Fmax, rows = F * (size_t)L;
+  const size_t Mp = e->Mp;
 
   // ---- weights
   {
     size_t off = 0;
     auto take = [&](size_t n) { size_t o = off; off += n; return o; };
-    e->off_patch_w = take((size_t)P * D); e->off_patch_b = take(D); e->off_pos = take((size_t)L * D);
     e->lo.resize(config->num_layers);
-    for (auto& o : e->lo) {
-      o.ln1_g = take(D); o.ln1_b = take(D); o.wqkv = take(D * 3 * D); o.bqkv = take(3 * D);
-      o.wo = take(D * D); o.bo = take(D); o.ln2_g = take(D); o.ln2_b = take(D);
-      o.w1 = take(D * M); o.b1 = take(M); o.w2 = take(M * D); o.b2 = take(D);
+    if (e->arch == 1) {
+      e->off_patch_w = take((size_t)P * D);
+      for (auto& o : e->lo) {
+        o.ln1_g = take(D); o.ln1_b = 0; o.wqkv = take(D * 3 * D); o.bqkv = take(3 * D);
+        o.wo = take(D * D); o.bo = take(D); o.ln2_g = take(D); o.ln2_b = 0;
+        o.w1 = take(D * 2 * M); o.b1 = take(2 * M); o.w2 = take(M * D); o.b2 = take(D);
+      }
+      e->off_post_g = take(D);
+    } else {
+      e->off_patch_w = take((size_t)P * D); e->off_patch_b = take(D); e->off_pos = take((size_t)L * D);
+      for (auto& o : e->lo) {
+        o.ln1_g = take(D); o.ln1_b = take(D); o.wqkv = take(D * 3 * D); o.bqkv = take(3 * D);
+        o.wo = take(D * D); o.bo = take(D); o.ln2_g = take(D); o.ln2_b = take(D);
+        o.w1 = take(D * M); o.b1 = take(M); o.w2 = take(M * D); o.b2 = take(D);
+      }
+      e->off_post_g = take(D); e->off_post_b = take(D);
     }
-    e->off_post_g = take(D); e->off_post_b = take(D);
   }
   if ((st = dalloc(e, &e->w_blob, weights->count)) != ET_OK) return bail(st);
   if (cudaMemcpy(e->w_blob, weights->data, weights->count * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
@@ -511,7 +587,42 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   } while (0)
   ET_A(e->X[0], rows * D * 4); ET_A(e->X[1], rows * D * 4);
   ET_A(e->Pm, rows * e->Kp * es); ET_A(e->Xn, rows * D * es); ET_A(e->QKV, rows * 3 * D * es);
-  ET_A(e->O, rows * D * es); ET_A(e->Hm, rows * M * es);
+  ET_A(e->O, rows * D * es); ET_A(e->Hm, rows * Mp * es);
+  if (e->arch == 1) {
+    ET_A(e->GU, rows * 2 * Mp * es);
+    ET_A(e->zeros, std::max(D, 2 * Mp) * 4);
+    ET_A(e->n_windows, 4);
+    cudaMemset(e->GU, 0, rows * 2 * Mp * es);
+    cudaMemset(e->zeros, 0, std::max(D, 2 * Mp) * 4);
+    // rotary table and token orders.  Internal order = window-major (windows row-major over the grid, tokens
+    // row-major inside a window), so that a window is a run of Lw consecutive rows; raster order otherwise.
+    std::vector<int> i2r(L), r2i(L);
+    for (int l = 0; l < L; ++l) i2r[l] = l;
+    if (e->ws > 0) {
+      const int ws = e->ws, wr = g / ws;
+      for (int l = 0; l < L; ++l) {
+        const int win = l / (ws * ws), in = l % (ws * ws);
+        i2r[l] = ((win / wr) * ws + in / ws) * g + (win % wr) * ws + in % ws;
+      }
+      ET_A(e->int2raster, (size_t)L * 4); ET_A(e->raster2int, (size_t)L * 4);
+      for (int l = 0; l < L; ++l) r2i[i2r[l]] = l;
+      cudaMemcpy(e->int2raster, i2r.data(), (size_t)L * 4, cudaMemcpyHostToDevice);
+      cudaMemcpy(e->raster2int, r2i.data(), (size_t)L * 4, cudaMemcpyHostToDevice);
+      e->r2i_host = r2i;
+    }
+    const int half = e->dh / 2, quarter = e->dh / 4;
+    std::vector<float2> tab((size_t)L * half);
+    for (int l = 0; l < L; ++l) {
+      const int gy = i2r[l] / g, gx = i2r[l] % g;
+      for (int i = 0; i < half; ++i) {
+        const double freq = pow((double)config->rope_theta, -2.0 * (double)(i % quarter) / (double)half);
+        const double ang = (double)(i < quarter ? gy : gx) * freq;
+        tab[(size_t)l * half + i] = make_float2((float)cos(ang), (float)sin(ang));
+      }
+    }
+    ET_A(e->rope_table, tab.size() * sizeof(float2));
+    cudaMemcpy(e->rope_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice);
+  }
   ET_A(e->lse, F * config->heads * L * 4); ET_A(e->score_partial, F * config->heads * L * 4);
   ET_A(e->scores, rows * 4); ET_A(e->simbuf, F * 4);
   for (int i = 0; i < 2; ++i) {
@@ -537,21 +648,25 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   if ((st = halloc(e, &e->h_tr_f, 2 * ET_MAX_MERGE_LAYERS * F)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_tr_b, 2 * ET_MAX_MERGE_LAYERS * F)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_scores, rows)) != ET_OK) return bail(st);
+  if (e->raster2int && (st = halloc(e, &e->h_scores_int, rows)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_keep, rows)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_video_kw, 2 * (size_t)e->Vmax)) != ET_OK) return bail(st);
   // zero the activation buffers once: rows beyond the live count are read (never stored) by tile loads
   cudaMemset(e->Pm, 0, rows * e->Kp * es); cudaMemset(e->Xn, 0, rows * D * es); cudaMemset(e->O, 0, rows * D * es);
-  cudaMemset(e->Hm, 0, rows * M * es); cudaMemset(e->QKV, 0, rows * 3 * D * es);
+  cudaMemset(e->Hm, 0, rows * Mp * es); cudaMemset(e->QKV, 0, rows * 3 * D * es);
   cudaMemset(e->sim_acc, 0, (size_t)similarity_plan_words(e->Fmax) * 8);
 
   if (e->bf) {
     // transposed bf16 copies of the dense weights ([out][in], K contiguous) + their tensor maps
     const char* err = nullptr;
-    auto convert = [&](size_t off, int K, int N, int k_pad, bf16** dst) -> et_status {
-      et_status s2 = dalloc(e, dst, (size_t)N * k_pad);
+    // rows_out > N: the N source columns land in rows [0, split) and [split + shift, ...), the rest stays zero
+    auto convert = [&](size_t off, int K, int N, int k_pad, bf16** dst, int rows_out = 0, int split = 0, int shift = 0) -> et_status {
+      if (rows_out <= 0) { rows_out = N; split = N; shift = 0; }
+      et_status s2 = dalloc(e, dst, (size_t)rows_out * k_pad);
       if (s2 != ET_OK) return s2;
+      if (rows_out != N && cudaMemset(*dst, 0, (size_t)rows_out * k_pad * sizeof(bf16)) != cudaSuccess) return ET_ERR_CUDA;
       ET_COUNT_LAUNCH();
-      transpose_to_bf16_kernel<<<dim3(cdiv(N, 32), cdiv(k_pad, 32)), dim3(32, 8)>>>(e->w_blob + off, *dst, K, N, k_pad);
+      transpose_to_bf16_kernel<<<dim3(cdiv(N, 32), cdiv(k_pad, 32)), dim3(32, 8)>>>(e->w_blob + off, *dst, K, N, k_pad, split, shift);
       return cudaGetLastError() == cudaSuccess ? ET_OK : ET_ERR_CUDA;
     };
     if ((st = convert(e->off_patch_w, P, (int)D, e->Kp, &e->patch_w_t)) != ET_OK) return bail(st);
@@ -562,19 +677,38 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
       const LayerOffsets& o = e->lo[i];
       if ((st = convert(o.wqkv, (int)D, (int)(3 * D), (int)D, &b.wqkv_t)) != ET_OK) return bail(st);
       if ((st = convert(o.wo, (int)D, (int)D, (int)D, &b.wo_t)) != ET_OK) return bail(st);
-      if ((st = convert(o.w1, (int)D, (int)M, (int)D, &b.w1_t)) != ET_OK) return bail(st);
-      if ((st = convert(o.w2, (int)M, (int)D, (int)M, &b.w2_t)) != ET_OK) return bail(st);
+      if (e->arch == 1) {
+        // [gate | up]: 2M source columns -> 2*Mp rows, each half padded to Mp; down: K padded to Mp
+        if ((st = convert(o.w1, (int)D, (int)(2 * M), (int)D, &b.w1_t, (int)(2 * Mp), (int)M, (int)(Mp - M))) != ET_OK) return bail(st);
+        if ((st = convert(o.w2, (int)M, (int)D, (int)Mp, &b.w2_t)) != ET_OK) return bail(st);
+      } else {
+        if ((st = convert(o.w1, (int)D, (int)M, (int)D, &b.w1_t)) != ET_OK) return bail(st);
+        if ((st = convert(o.w2, (int)M, (int)D, (int)M, &b.w2_t)) != ET_OK) return bail(st);
+      }
       bool ok = make_tma_weight(&b.d_wqkv, b.wqkv_t, 3 * D, D, &err) &&
                 make_tma_weight(&b.d_wo, b.wo_t, D, D, &err) &&
-                make_tma_weight(&b.d_w1, b.w1_t, M, D, &err) &&
-                make_tma_weight(&b.d_w2, b.w2_t, D, M, &err);
+                make_tma_weight(&b.d_w1, b.w1_t, e->arch == 1 ? 2 * Mp : M, D, &err) &&
+                make_tma_weight(&b.d_w2, b.w2_t, D, Mp, &err);
       if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
     }
     bool ok = make_tma_2d_bf16(&e->d_Pm, e->Pm, rows, e->Kp, 128, &err) && make_tma_2d_bf16(&e->d_Xn, e->Xn, rows, D, 128, &err) &&
-              make_tma_2d_bf16(&e->d_O, e->O, rows, D, 128, &err) && make_tma_2d_bf16(&e->d_Hm, e->Hm, rows, M, 128, &err) &&
+              make_tma_2d_bf16(&e->d_O, e->O, rows, D, 128, &err) && make_tma_2d_bf16(&e->d_Hm, e->Hm, rows, Mp, 128, &err) &&
               make_tma_out(&e->c_X[0], e->X[0], rows, D, true, &err) && make_tma_out(&e->c_X[1], e->X[1], rows, D, true, &err) &&
-              make_tma_out(&e->c_QKV, e->QKV, rows, 3 * D, false, &err) && make_tma_out(&e->c_Hm, e->Hm, rows, M, false, &err);
+              make_tma_out(&e->c_QKV, e->QKV, rows, 3 * D, false, &err) && make_tma_out(&e->c_Hm, e->Hm, rows, Mp, false, &err);
+    if (ok && e->arch == 1) ok = make_tma_out(&e->c_GU, e->GU, rows, 2 * Mp, false, &err);
     if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
+    if (e->arch == 1) {
+      // gate | up biases in the padded layout
+      std::vector<float> hb((size_t)config->num_layers * 2 * Mp, 0.f);
+      for (int i = 0; i < config->num_layers; ++i) {
+        const float* src = weights->data + e->lo[i].b1;
+        float* dst = hb.data() + (size_t)i * 2 * Mp;
+        memcpy(dst, src, M * sizeof(float));
+        memcpy(dst + Mp, src + M, M * sizeof(float));
+      }
+      if ((st = dalloc(e, &e->bgu_pad, hb.size())) != ET_OK) return bail(st);
+      if (cudaMemcpy(e->bgu_pad, hb.data(), hb.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) return bail(ET_ERR_CUDA);
+    }
     if (attention_tc_supported(e->dh)) {
       if (!make_attention_maps(&e->attn_maps, (const bf16*)e->QKV, (long long)rows, config->heads, e->dh))
         return bail(fail(e, ET_ERR_CUDA, "tensor map of the attention operands"));
@@ -610,11 +744,11 @@ et_status et_encode_batch_host(et_encoder* e, const float* frames_host, const in
                                const et_params* params, void* cuda_stream, const et_host_buffers* dst, et_result* out) {
   if (!e || !frames_host || !video_offsets_host || !dst || !out) return fail(e, ET_ERR_INVALID_ARG, "null argument");
   if (V < 1 || V > e->Vmax) return fail(e, ET_ERR_CAPACITY, "number of videos outside [1, max_videos]");
-  const int T = video_offsets_host[V];
-  if (T < 1 || T > e->Fmax) return fail(e, ET_ERR_CAPACITY, "frames outside [1, max_frames_total]");
+  const int T = video_offsets_host[V];                     // input frames
+  if (T < 1 || T > e->Fmax * e->tp) return fail(e, ET_ERR_CAPACITY, "frames outside [1, max_frames_total]");
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const size_t frame_floats = (size_t)3 * e->cfg.image_size * e->cfg.image_size;
-  if (!e->frames_stage) ET_TRY(dalloc(e, &e->frames_stage, (size_t)e->Fmax * frame_floats));
+  if (!e->frames_stage) ET_TRY(dalloc(e, &e->frames_stage, (size_t)e->Fmax * e->tp * frame_floats));
   ET_CUDA(e, cudaMemcpyAsync(e->frames_stage, frames_host, (size_t)T * frame_floats * sizeof(float), cudaMemcpyHostToDevice, s));
   et_result r{};
   ET_TRY(encode_impl(e, e->frames_stage, video_offsets_host, V, params, s, &r));

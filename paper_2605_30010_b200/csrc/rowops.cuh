@@ -97,6 +97,29 @@ __device__ __forceinline__ void layernorm_row_inplace(float4 (&v)[NV], int D, in
   }
 }
 
+// y = x / sqrt(mean(x^2) + eps) * g
+template <int NV>
+__device__ __forceinline__ void rmsnorm_row_inplace(float4 (&v)[NV], int D, int lane, const float* __restrict__ g,
+                                                    float eps) {
+  const int nvec = D >> 2;
+  float q = 0.f;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) q += (v[j].x * v[j].x + v[j].y * v[j].y) + (v[j].z * v[j].z + v[j].w * v[j].w);   // padding chunks are zero
+  const float r = rsqrtf(warp_sum(q) / (float)D + eps);
+  const float4* g4 = reinterpret_cast<const float4*>(g);
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    const int i = lane + 32 * j;
+    if (i < nvec) {
+      const float4 gg = __ldg(g4 + i);
+      v[j].x = v[j].x * r * gg.x;
+      v[j].y = v[j].y * r * gg.y;
+      v[j].z = v[j].z * r * gg.z;
+      v[j].w = v[j].w * r * gg.w;
+    }
+  }
+}
+
 __device__ __forceinline__ float gelu_f(float x, int tanh_approx) {
   if (tanh_approx) {
     const float c = 0.7978845608028654f;   // sqrt(2/pi)

@@ -84,8 +84,8 @@ __global__ void __launch_bounds__(256) select_video_tokens_kernel(SelectArgs a) 
     }
     sh_v = lo;
   }
-  const float* sc = a.scores + (size_t)f * a.L;
-  for (int j = threadIdx.x; j < a.L; j += blockDim.x) sh_a[j] = nan_to_lowest(sc[j]);
+  const float* sc = a.scores + (size_t)f * a.L;      // in the encoder's internal token order; selection is in raster order
+  for (int j = threadIdx.x; j < a.L; j += blockDim.x) sh_a[j] = nan_to_lowest(sc[a.raster2int ? a.raster2int[j] : j]);
   __syncthreads();
   const int v = sh_v, L = a.L;
   ET_CHECK(v >= 0 && v < a.n_videos && a.fl.vid_off[v] <= f && f < a.fl.vid_off[v + 1], return);
@@ -248,7 +248,7 @@ __global__ void __launch_bounds__(256)
 gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restrict__ keep, const int* __restrict__ count,
                      int* __restrict__ frame_offsets, int* __restrict__ totals, int n_cap, int L, int D,
                      const float* __restrict__ ln_g, const float* __restrict__ ln_b, float eps, float* __restrict__ tokens,
-                     int* __restrict__ token_pos, const int* __restrict__ n_frames_dev) {
+                     int* __restrict__ token_pos, const int* __restrict__ n_frames_dev, const int* __restrict__ raster2int) {
   extern __shared__ unsigned short sh_pos[];   // [L] position of the r-th kept token of this frame
   __shared__ int sh_before[8], sh_wkept[8];
   const int n = n_frames_dev ? min(*n_frames_dev, n_cap) : n_cap;
@@ -302,8 +302,9 @@ gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restric
     const int j = sh_pos[r];
     ET_CHECK(j < L, continue);
     float4 v[NV];
-    load_row<NV>(x + ((size_t)f * L + j) * D, D, lane, v);
-    if (ln_g) layernorm_row_inplace<NV>(v, D, lane, ln_g, ln_b, eps);
+    load_row<NV>(x + ((size_t)f * L + (raster2int ? raster2int[j] : j)) * D, D, lane, v);   // the row of raster position j
+    if (ln_g && ln_b) layernorm_row_inplace<NV>(v, D, lane, ln_g, ln_b, eps);
+    else if (ln_g) rmsnorm_row_inplace<NV>(v, D, lane, ln_g, eps);
     store_row<NV>(tokens + (size_t)(out0 + r) * D, D, lane, v);
     if (lane == 0) token_pos[out0 + r] = j;
   }
@@ -311,14 +312,14 @@ gather_tokens_kernel(const float* __restrict__ x, const unsigned char* __restric
 
 void launch_gather_tokens(const float* x, const unsigned char* keep, const int* count, int* frame_offsets, int* totals,
                           int n_cap, int L, int D, const float* ln_g, const float* ln_b, float eps, float* tokens,
-                          int* token_pos, const int* n_frames_dev, cudaStream_t s) {
+                          int* token_pos, const int* n_frames_dev, cudaStream_t s, const int* raster2int) {
   if (n_cap <= 0) return;
   const int slices = max(1, min(16, cdiv(L, 64)));
   ET_COUNT_LAUNCH();
   const int need = cdiv(D / 4, 32);      // float4 chunks per lane
 #define ET_GATHER(NV)                                                                                      \
   gather_tokens_kernel<NV><<<dim3(slices, n_cap), 256, sizeof(unsigned short) * L, s>>>(                   \
-      x, keep, count, frame_offsets, totals, n_cap, L, D, ln_g, ln_b, eps, tokens, token_pos, n_frames_dev)
+      x, keep, count, frame_offsets, totals, n_cap, L, D, ln_g, ln_b, eps, tokens, token_pos, n_frames_dev, raster2int)
   if (need <= 2) ET_GATHER(2);
   else if (need <= 4) ET_GATHER(4);
   else if (need <= 6) ET_GATHER(6);

@@ -215,3 +215,52 @@ def test_launch_counter_and_reproducibility(B):
     b = enc.encode_batch(to_cuda(frames), offs, wl.params)
     assert torch.equal(a.tokens, b.tokens) and torch.equal(a.token_pos, b.token_pos)
     enc.close()
+
+
+# ------------------------------------------------------------------ Qwen2.5-VL-style encoder (windows, 2-D rotary positions)
+
+def test_qwenvl_tiny_fp32(B):
+    err, log = run_workload(B, workload("qwenvl_tiny"), np.float64, F32_TOL, F32_SIM, F32_SCORE)
+    assert not log
+
+
+def test_qwenvl_tiny_fp32_uncompressed_and_full_attention_only(B):
+    wl = workload("qwenvl_tiny")
+    run_workload(B, wl.uncompressed(), np.float64, F32_TOL, F32_SIM, F32_SCORE)
+    nowin = dataclasses.replace(wl, shape=dataclasses.replace(wl.shape, window=0, full_attn_layers=()))
+    run_workload(B, nowin, np.float64, F32_TOL, F32_SIM, F32_SCORE)
+
+
+def test_qwenvl_fp32_ragged_batch_three_frames_per_patch(B):
+    shape = EncoderShape(image_size=84, patch_size=14, num_layers=4, hidden=48, heads=3, mlp_dim=52, arch=1,
+                         temporal_patch=3, window=3, full_attn_layers=(0, 3))
+    vids = (VideoSpec(15, 0.05, 1), VideoSpec(3, 0.2, 2), VideoSpec(27, 0.03, 3))
+    p = MergeParams(merge_layers=(1, 3), tau_seg=0.55, tau_merge=0.6, selection=1, retain_mode=1, retain=0.4)
+    wl = Workload("qwenvl_ragged", shape, "f32", vids, p, 78)
+    run_workload(B, wl, np.float64, F32_TOL, F32_SIM, F32_SCORE)
+
+
+def test_qwenvl_small_bf16(B):
+    """Head dim 80 and an MLP width that is padded on the tensor-core path (200 -> 256)."""
+    shape = EncoderShape(image_size=112, patch_size=14, num_layers=4, hidden=160, heads=2, mlp_dim=200, arch=1,
+                         temporal_patch=2, window=4, full_attn_layers=(1, 3))
+    vids = (VideoSpec(24, 0.03, 1), VideoSpec(14, 0.1, 2))
+    p = MergeParams(merge_layers=(1, 3), tau_seg=0.5, tau_merge=0.6, selection=1, retain_mode=1, retain=0.3)
+    wl = Workload("qwenvl_small_bf16", shape, "bf16", vids, p, 6)
+    run_workload(B, wl, np.float64, BF16_TOL, BF16_SIM, BF16_SCORE)
+
+
+def test_qwenvl_argument_errors(B):
+    wl = workload("qwenvl_tiny")
+    frames, offs = make_batch(wl)
+    blob = make_weights(wl.shape, wl.weight_seed)
+    for bad in (dict(window=3), dict(full_attn_layers=(1,)), dict(heads=32)):      # grid 4 % 3, last block windowed, head dim 2
+        with pytest.raises(B.EarlyTomError) as ei:
+            shape = dataclasses.replace(wl.shape, **bad)
+            B.Encoder(shape, make_weights(shape, 1), B.ET_F32, 24)
+        assert ei.value.status == 2
+    enc = B.Encoder(wl.shape, blob, B.ET_F32, 24)
+    with pytest.raises(B.EarlyTomError) as ei:
+        enc.encode_batch(to_cuda(frames[:5]), [0, 5], wl.params)                    # 5 frames: not a multiple of 2
+    assert ei.value.status == 1
+    enc.close()
