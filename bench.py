@@ -432,7 +432,7 @@ def main():
     # input from L2.
     V = len(wl.videos)
     T = wl.total_frames
-    n_rot = 4 if V == 1 else 2
+    n_rot = 4 if (V == 1 and T <= 64) else 2
     sets = []
     for sd in rank_video_seeds(rank, n_rot):
         vs = [make_video(v.n_frames, shape.image_size, shape.patch_size, v.resample_p, v.seed + sd, v.jitter, v.cut_every) for v in wl.videos]
@@ -551,8 +551,11 @@ def main():
                        "merge_layers": list(params.merge_layers), "tau_seg": params.tau_seg, "tau_merge": params.tau_merge,
                        "retain": params.retain, "window_mode": params.window_mode,
                        "frames_per_block": res.frames_per_block, "frames_out": res.n_frames_out,
-                       "stage1_frames_out": res.n_frames_out, "stage1_frame_retention": round(res.n_frames_out / T, 4),
-                       "tokens_out": res.n_tokens, "retained_ratio": round(res.n_tokens / (T * shape.tokens_per_frame), 4),
+                       "encoder_frames": T // shape.temporal_patch,
+                       "stage1_frames_out": res.n_frames_out,
+                       "stage1_frame_retention": round(res.n_frames_out / (T // shape.temporal_patch), 4),
+                       "tokens_out": res.n_tokens,
+                       "retained_ratio": round(res.n_tokens / ((T // shape.temporal_patch) * shape.tokens_per_frame), 4),
                        "parallelism": f"replicas x{world}",
                        "l2": f"inputs rotate over {n_rot} videos; weights (824 MB) + activations per step exceed the 126 MB L2"},
             "ms_per_video": ms_step, "clocks": clocks, "gpu_launches": int(launches),

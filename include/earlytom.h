@@ -320,8 +320,8 @@ ET_API et_status et_gather_tokens(const float* x_dev, const unsigned char* keep_
  * a multiple of 16); epilogue 0: store bf16; 1: GELU then store bf16; 2: c fp32 += result
  * (residual, in place); 3: c fp32 = result + table[(row % table_rows)][N] (position embedding);
  * 4: gated feed-forward of the language model (earlytom_llm.h): the rows of w are ordered in tiles of
- * 256 = four groups of (32 gate rows, 32 up rows) of the same 32 outputs, bias is ignored, N % 256 == 0 and
- * c is bf16 [M][N/2] = silu(gate) * up.
+ * 256 = four groups of (32 gate rows, 32 up rows) of the same 32 outputs, bias [N] follows the same order, N % 256 == 0
+ * and c is bf16 [M][N/2] = silu(gate + bias) * (up + bias).
  * status_dev int [1] receives a non-zero code if a bounded wait expired. */
 ET_API et_status et_linear_bf16(const void* a_dev, const void* w_dev, const float* bias_dev, void* c_dev, int M, int N,
                          int K, int epilogue, int gelu_tanh, const float* table_dev, int table_rows,
@@ -332,6 +332,12 @@ ET_API et_status et_linear_bf16(const void* a_dev, const void* w_dev, const floa
  * lse_dev fp32 [n][heads][L] receives the row log-sum-exp (natural log, of the scaled logits). */
 ET_API et_status et_attention(const void* qkv_dev, void* out_dev, float* lse_dev, int n, int L, int heads, int head_dim,
                        int dtype, void* cuda_stream);
+
+/* The same inside windows (the Qwen2.5-VL-style encoder of et_config.arch 1): the rows of a frame are ordered so that a
+ * window is a run of window_rows consecutive rows (window_rows divides L), and a query attends only to the keys of its
+ * own window.  lse_scratch_dev fp32 [n][heads][L] is overwritten with values whose layout is not specified. */
+ET_API et_status et_attention_windowed(const void* qkv_dev, void* out_dev, float* lse_scratch_dev, int n, int L, int heads,
+                                int head_dim, int window_rows, int dtype, void* cuda_stream);
 
 /* Per-token attention score of Alg. 2's input A: score[f][j] = mean over heads and queries of
  * softmax(QK^T/sqrt(d))[q][j], recomputed from qkv_dev and lse_dev.  partial_dev fp32

@@ -157,6 +157,7 @@ def load_library(path: str = _LIB_PATH) -> C.CDLL:
     lib.et_gather_tokens.argtypes = [vp, vp, i, i, i, vp, vp, f, vp, C.c_size_t, vp, vp, _I32P, vp]
     lib.et_linear_bf16.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, i, vp, vp]
     lib.et_attention.argtypes = [vp, vp, vp, i, i, i, i, i, vp]
+    lib.et_attention_windowed.argtypes = [vp, vp, vp, i, i, i, i, i, i, vp]
     lib.et_attention_scores.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp]
     lib.et_layernorm.argtypes = [vp, vp, vp, f, vp, i, i, i, vp]
     lib.et_llm_create.argtypes = [C.POINTER(et_llm_config), C.POINTER(et_llm_weights), C.POINTER(vp)]
@@ -552,6 +553,16 @@ def et_linear_bf16(a, w, bias, epilogue=0, gelu_tanh=1, c=None, table=None, stre
                                 _ptr(table), int(table.shape[0]) if table is not None else 0, _ptr(status),
                                 _stream_ptr(stream)))
     return c, status
+
+
+def et_attention_windowed(qkv, n, L, heads, head_dim, window_rows, stream=None):
+    import torch
+    dtype = ET_BF16 if qkv.dtype == torch.bfloat16 else ET_F32
+    out = torch.empty((n * L, heads * head_dim), dtype=qkv.dtype, device=qkv.device)
+    lse = torch.empty((n, heads, L), dtype=torch.float32, device=qkv.device)
+    _check(lib().et_attention_windowed(_ptr(qkv), _ptr(out), _ptr(lse), n, L, heads, head_dim, int(window_rows), dtype,
+                                       _stream_ptr(stream)))
+    return out
 
 
 def et_attention(qkv, n, L, heads, head_dim, stream=None):

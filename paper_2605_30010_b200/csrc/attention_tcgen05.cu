@@ -15,10 +15,15 @@
 // domain), so the rescale of O in TMEM is rare; P stays below 2^8, which bf16 represents without loss
 // of relative precision.  The final division by the row sum makes the result independent of that choice.
 //
-// Head dim 64 or 72.  A head row is 64 elements (one 128-byte swizzled row) plus, for 72, a tail of 8
-// elements: for Q and K a separate 16-byte-per-row tile whose contraction step pairs it with a block of
-// zeros (K = 16 for the MMA); for V a second swizzled 64-column box, so that O += P V is one MMA of N = 80
-// per 16 keys (its columns 72..79 are never read).  Global memory keeps the packed [tokens][3*D] layout.
+// Head dim 64, 72 or 80.  A head row is 64 elements (one 128-byte swizzled row) plus a tail of 8 or 16 elements:
+// for Q and K the tail is one contraction step (K = 16) made of two 16-byte-per-row column blocks, the second of
+// which is a block of zeros for head dim 72 and the elements 72..79 for head dim 80; for V a second swizzled
+// 64-column box, so that O += P V is one MMA of N = 80 per 16 keys (columns beyond the head are never read).
+// Global memory keeps the packed [tokens][3*D] layout.
+//
+// Windowed attention (window_rows > 0): the tokens of a frame are ordered so that a window is a run of window_rows
+// consecutive rows; the kernel sweeps the whole frame as usual and the softmax masks the keys outside the query's
+// window (a tile without any key of the window contributes zeros).
 #include "common.cuh"
 #include "softmax_tile.cuh"
 #include "tcgen05.cuh"
@@ -53,9 +58,10 @@ constexpr int OFF_Q_MAIN = 0;
 constexpr int OFF_K_MAIN = OFF_Q_MAIN + 2 * MAIN_BYTES;
 constexpr int V_STAGE_BYTES = 2 * MAIN_BYTES;                   // columns 0..63 of the head, then the 64 columns from 64 on
 constexpr int OFF_V_MAIN = OFF_K_MAIN + KV_STAGES * MAIN_BYTES;
+constexpr int TAIL_SLOT = 2 * TAIL_BYTES;                       // two column blocks (elements 64..71, 72..79) per Q group / K stage
 constexpr int OFF_Q_TAIL = OFF_V_MAIN + KV_STAGES * V_STAGE_BYTES;
-constexpr int OFF_K_TAIL = OFF_Q_TAIL + 2 * TAIL_BYTES;
-constexpr int OFF_ZERO = OFF_K_TAIL + KV_STAGES * TAIL_BYTES;   // 2 KB of zeros: the second half of the Q K^T tail step
+constexpr int OFF_K_TAIL = OFF_Q_TAIL + 2 * TAIL_SLOT;
+constexpr int OFF_ZERO = OFF_K_TAIL + KV_STAGES * TAIL_SLOT;    // 2 KB of zeros: the second half of the tail step for head dim 72
 constexpr int OFF_BARS = OFF_ZERO + TAIL_BYTES;
 constexpr int ATT_SMEM_BYTES = OFF_BARS + 256 + 1024;
 
@@ -64,6 +70,7 @@ constexpr int B_Q_FULL = 0, B_K_FULL = 1, B_V_FULL = B_K_FULL + KV_STAGES, B_KV_
               B_S_FULL = B_KV_EMPTY + KV_STAGES, B_P_FULL = B_S_FULL + 2, B_O_READY = B_P_FULL + 2, B_Q_EMPTY = B_O_READY + 2,
               B_COUNT = B_Q_EMPTY + 1;
 static_assert(B_COUNT * 8 + 8 <= 256, "barrier area");
+static_assert(ATT_SMEM_BYTES <= 232448, "shared memory");
 
 // TMEM columns: S of group t at t*128 (P aliases its first 64 columns), O of group t at 256 + t*80
 constexpr int TMEM_COLS = 512;
@@ -75,13 +82,15 @@ struct AttnArgs {
   int n_cap, L, heads;
   const int* n_frames_dev;
   int* status;
+  int window_rows;       // 0, or the rows of an attention window (a divisor of L)
 };
 
 template <int DH>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_constant__ CUtensorMap tma_tail, AttnArgs g) {
   constexpr bool HAS_TAIL = DH > 64;
-  static_assert(DH == 64 || DH == 72, "head dim");
+  constexpr bool TAIL2 = DH > 72;                    // the second column block of the tail step holds elements 72..79
+  static_assert(DH == 64 || DH == 72 || DH == 80, "head dim");
   const int n = g.n_frames_dev ? min(*g.n_frames_dev, g.n_cap) : g.n_cap;
   const int L = g.L, D = g.heads * DH;
   const int n_tiles = (L + KT - 1) / KT;
@@ -140,7 +149,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_main) : "memory");
       if (HAS_TAIL) asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_tail) : "memory");
-      constexpr uint32_t TILE_TX = MAIN_BYTES + (HAS_TAIL ? TAIL_BYTES : 0);
+      constexpr uint32_t TILE_TX = MAIN_BYTES + (HAS_TAIL ? TAIL_BYTES : 0) + (TAIL2 ? TAIL_BYTES : 0);
       bool ok = true;
       int gt = 0;                                        // key tiles loaded so far: ring stage and phase
       for (int i = 0; i < my_items && ok; ++i) {
@@ -152,7 +161,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
         mbar_arrive_expect_tx(bar(B_Q_FULL), 2 * TILE_TX);
         for (int t = 0; t < 2; ++t) {
           tma_load_2d(base + OFF_Q_MAIN + t * MAIN_BYTES, &tma_main, bar(B_Q_FULL), h * DH, row_base + q0 + t * QT);
-          if (HAS_TAIL) tma_load_2d(base + OFF_Q_TAIL + t * TAIL_BYTES, &tma_tail, bar(B_Q_FULL), h * DH + 64, row_base + q0 + t * QT);
+          if (HAS_TAIL) tma_load_2d(base + OFF_Q_TAIL + t * TAIL_SLOT, &tma_tail, bar(B_Q_FULL), h * DH + 64, row_base + q0 + t * QT);
+          if (TAIL2) tma_load_2d(base + OFF_Q_TAIL + t * TAIL_SLOT + TAIL_BYTES, &tma_tail, bar(B_Q_FULL), h * DH + 72, row_base + q0 + t * QT);
         }
         for (int j = 0; j < n_tiles; ++j, ++gt) {
           const int s = gt % KV_STAGES;
@@ -161,7 +171,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
           const int y = row_base + j * KT;
           mbar_arrive_expect_tx(bar(B_K_FULL + s), TILE_TX);
           tma_load_2d(base + OFF_K_MAIN + s * MAIN_BYTES, &tma_main, bar(B_K_FULL + s), D + h * DH, y);
-          if (HAS_TAIL) tma_load_2d(base + OFF_K_TAIL + s * TAIL_BYTES, &tma_tail, bar(B_K_FULL + s), D + h * DH + 64, y);
+          if (HAS_TAIL) tma_load_2d(base + OFF_K_TAIL + s * TAIL_SLOT, &tma_tail, bar(B_K_FULL + s), D + h * DH + 64, y);
+          if (TAIL2) tma_load_2d(base + OFF_K_TAIL + s * TAIL_SLOT + TAIL_BYTES, &tma_tail, bar(B_K_FULL + s), D + h * DH + 72, y);
           // V: a second 64-column box starting at column 64 of the head; only its first 8 columns belong to
           // the head, the rest (the next head, or zeros past the row end) lands in output columns nobody reads
           mbar_arrive_expect_tx(bar(B_V_FULL + s), HAS_TAIL ? V_STAGE_BYTES : MAIN_BYTES);
@@ -183,11 +194,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
       const uint32_t zero = base + OFF_ZERO;
       const uint64_t q_main0 = smem_desc(base + OFF_Q_MAIN, 16, 1024, 2), k_main0 = smem_desc(base + OFF_K_MAIN, 16, 1024, 2),
                      v_main0 = smem_desc(base + OFF_V_MAIN, MAIN_BYTES, 1024, 2);
-      const uint64_t q_tail0 = smem_desc(base + OFF_Q_TAIL, zero - (base + OFF_Q_TAIL), 128, 0),
-                     k_tail0 = smem_desc(base + OFF_K_TAIL, zero - (base + OFF_K_TAIL), 128, 0);
-      constexpr uint64_t MAIN_STEP = MAIN_BYTES >> 4, TAIL_STEP = TAIL_BYTES >> 4;
+      // the second column block of a tail: the slot's own second block (head dim 80) or the shared block of zeros
+      const uint64_t q_tail0 = smem_desc(base + OFF_Q_TAIL, TAIL2 ? (uint32_t)TAIL_BYTES : zero - (base + OFF_Q_TAIL), 128, 0),
+                     k_tail0 = smem_desc(base + OFF_K_TAIL, TAIL2 ? (uint32_t)TAIL_BYTES : zero - (base + OFF_K_TAIL), 128, 0);
+      constexpr uint64_t MAIN_STEP = MAIN_BYTES >> 4, TAIL_STEP = TAIL_SLOT >> 4;
       auto main_desc = [&](uint64_t d0, int i) { return d0 + (uint64_t)i * MAIN_STEP; };
-      auto tail_desc = [&](uint64_t d0, int i, int off_shift) { return d0 + (uint64_t)i * TAIL_STEP - (((uint64_t)i * TAIL_STEP) << off_shift); };
+      // slot i: the address moves on by i slots; the distance to the shared zero block shrinks by as much
+      auto tail_desc = [&](uint64_t d0, int i, int off_shift) {
+        return d0 + (uint64_t)i * TAIL_STEP - (TAIL2 ? 0ull : (((uint64_t)i * TAIL_STEP) << off_shift));
+      };
       // Step g issues  O += P V  of key tile g-1 and  S = Q K^T  of key tile g (group 0, then group 1),
       // g counting the key tiles of all items of this CTA: the first Q K^T of an item overlaps the last
       // softmax of the item before it.
@@ -223,7 +238,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)                       // 16 elements = 32 bytes inside the swizzle row
               mma_ss_elect(tmem_base + t * 128, qd + 2 * ks, kd + 2 * ks, idesc, ks != 0 ? 1u : 0u);
-            // elements 64..71 and a block of zeros: two 8-element column blocks, the second one `lbo` bytes away
+            // elements 64..71 and 72..79 (or a block of zeros): two 8-element column blocks, the second one `lbo` bytes away
             if (HAS_TAIL) mma_ss_elect(tmem_base + t * 128, tail_desc(q_tail0, t, 16), tail_desc(k_tail0, s, 16), idesc, 1u);
             commit_elect(bar(B_S_FULL + t));
             if (t == 1 && j == n_tiles - 1) commit_elect(bar(B_Q_EMPTY));   // the item's last read of Q
@@ -264,15 +279,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
       if (nch > 1) tmem_regs_ready(r1);
       if (nch > 2) tmem_regs_ready(r2);
       if (nch > 3) tmem_regs_ready(r3);
-      const bool full = nk == KT;
+      // valid columns of this tile for this row: [lo, hi) (the keys of the row's window, or all nk keys)
+      int lo = 0, hi = nk;
+      if (g.window_rows > 0) {
+        const int w0 = (min(q, L - 1) / g.window_rows) * g.window_rows - j * KT;
+        lo = max(w0, 0);
+        hi = min(nk, w0 + g.window_rows);
+      }
+      const bool full = nk == KT && g.window_rows == 0;
       float mx;
       if (full) {
         mx = fmaxf(fmaxf(row_max<false>(r0, 0, nk), row_max<false>(r1, 32, nk)), fmaxf(row_max<false>(r2, 64, nk), row_max<false>(r3, 96, nk)));
       } else {
-        mx = row_max<true>(r0, 0, nk);
-        if (nch > 1) mx = fmaxf(mx, row_max<true>(r1, 32, nk));
-        if (nch > 2) mx = fmaxf(mx, row_max<true>(r2, 64, nk));
-        if (nch > 3) mx = fmaxf(mx, row_max<true>(r3, 96, nk));
+        mx = row_max<true>(r0, 0, hi, lo);
+        if (nch > 1) mx = fmaxf(mx, row_max<true>(r1, 32, hi, lo));
+        if (nch > 2) mx = fmaxf(mx, row_max<true>(r2, 64, hi, lo));
+        if (nch > 3) mx = fmaxf(mx, row_max<true>(r3, 96, hi, lo));
       }
       mx *= scale2;
       if (__any_sync(0xffffffffu, mx > m + RESCALE_GAP)) {
@@ -308,10 +330,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
         probs<false>(r2, 64, nk, scale2, m, ls, s_addr + 32);
         probs<false>(r3, 96, nk, scale2, m, ls, s_addr + 48);
       } else {
-        probs<true>(r0, 0, nk, scale2, m, ls, s_addr);
-        if (nch > 1) probs<true>(r1, 32, nk, scale2, m, ls, s_addr + 16);
-        if (nch > 2) probs<true>(r2, 64, nk, scale2, m, ls, s_addr + 32);
-        if (nch > 3) probs<true>(r3, 96, nk, scale2, m, ls, s_addr + 48);
+        probs<true>(r0, 0, hi, scale2, m, ls, s_addr, lo);
+        if (nch > 1) probs<true>(r1, 32, hi, scale2, m, ls, s_addr + 16, lo);
+        if (nch > 2) probs<true>(r2, 64, hi, scale2, m, ls, s_addr + 32, lo);
+        if (nch > 3) probs<true>(r3, 96, hi, scale2, m, ls, s_addr + 48, lo);
       }
       l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       tmem_wait_st();
@@ -342,15 +364,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tma_main, const __grid_c
         }
       }
       if (HAS_TAIL) {
-        uint32_t r[8];
-        tmem_ld8(o_addr + 64, r);
+        uint32_t r[16];
+        tmem_ld16(o_addr + 64, r);
         if (q < L) {
-          uint4 o;
-          o.x = pack_bf16(__uint_as_float(r[0]) * inv, __uint_as_float(r[1]) * inv);
-          o.y = pack_bf16(__uint_as_float(r[2]) * inv, __uint_as_float(r[3]) * inv);
-          o.z = pack_bf16(__uint_as_float(r[4]) * inv, __uint_as_float(r[5]) * inv);
-          o.w = pack_bf16(__uint_as_float(r[6]) * inv, __uint_as_float(r[7]) * inv);
-          *reinterpret_cast<uint4*>(orow + 64) = o;
+#pragma unroll
+          for (int i = 0; i < (TAIL2 ? 16 : 8); i += 8) {
+            uint4 o;
+            o.x = pack_bf16(__uint_as_float(r[i + 0]) * inv, __uint_as_float(r[i + 1]) * inv);
+            o.y = pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+            o.z = pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+            o.w = pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + 64 + i) = o;
+          }
         }
       }
       if (q < L) g.lse[((size_t)f * g.heads + h) * L + q] = (m + log2f(l)) * LN2;
@@ -417,7 +442,7 @@ cudaError_t run(const AttnMaps& maps, const AttnArgs& a, cudaStream_t s) {
 
 }  // namespace
 
-bool attention_tc_supported(int dh) { return dh == 64 || dh == 72; }
+bool attention_tc_supported(int dh) { return dh == 64 || dh == 72 || dh == 80; }
 
 bool make_attention_maps(AttnMaps* out, const bf16* qkv, long long rows, int heads, int dh) {
   if (!attention_tc_supported(dh)) return false;
@@ -429,9 +454,11 @@ bool make_attention_maps(AttnMaps* out, const bf16* qkv, long long rows, int hea
 }
 
 cudaError_t launch_attention_tc(const AttnMaps& maps, bf16* out, float* lse, int n_cap, int L, int heads, int dh,
-                                const int* n_frames_dev, int* status_dev, cudaStream_t s) {
+                                const int* n_frames_dev, int* status_dev, cudaStream_t s, int window_rows) {
   if (n_cap <= 0) return cudaSuccess;
-  AttnArgs a{out, lse, n_cap, L, heads, n_frames_dev, status_dev};
+  if (window_rows < 0 || (window_rows > 0 && L % window_rows != 0)) return cudaErrorInvalidValue;
+  AttnArgs a{out, lse, n_cap, L, heads, n_frames_dev, status_dev, window_rows == L ? 0 : window_rows};
+  if (dh == 80) return run<80>(maps, a, s);
   if (dh == 72) return run<72>(maps, a, s);
   if (dh == 64) return run<64>(maps, a, s);
   return cudaErrorInvalidValue;

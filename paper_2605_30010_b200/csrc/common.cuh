@@ -77,7 +77,7 @@ struct LayerTrace {
 };
 
 // EPI_SWIGLU: the N accumulator columns are pairs of 32-column chunks (gate, up) of the same 32 outputs; the layer
-// writes c [M][N/2] = silu(gate) * up in bf16 and takes no bias.  N % 256 == 0.
+// writes c [M][N/2] = silu(gate + bias) * (up + bias) in bf16, bias [N] in the order of the weight rows.  N % 256 == 0.
 enum Epilogue : int { EPI_STORE = 0, EPI_GELU = 1, EPI_RESIDUAL = 2, EPI_TABLE = 3, EPI_SWIGLU = 4 };
 
 // ---- elementwise.cu ------------------------------------------------------------------------
@@ -130,12 +130,14 @@ void launch_attention_f32(const float* qkv, float* out, float* lse, int n_cap, i
 void launch_attention_bf16(const bf16* qkv, bf16* out, float* lse, int n_cap, int L, int heads, int dh,
                            const int* n_frames_dev, cudaStream_t s);
 bool attention_bf16_supported(int L, int heads, int dh);
-// tcgen05 attention (attention_tcgen05.cu): head dims 64 and 72.  The maps describe qkv [rows][3*D] bf16.
+// tcgen05 attention (attention_tcgen05.cu): head dims 64, 72 and 80.  The maps describe qkv [rows][3*D] bf16.
 struct AttnMaps { TmaDesc main, tail; };
 bool attention_tc_supported(int dh);
 bool make_attention_maps(AttnMaps* out, const bf16* qkv, long long rows, int heads, int dh);
+// window_rows > 0: a query attends only to the keys of its run of window_rows consecutive rows of the frame
 cudaError_t launch_attention_tc(const AttnMaps& maps, bf16* out, float* lse, int n_cap, int L, int heads, int dh,
-                                const int* n_frames_dev, int* status_dev, cudaStream_t s);
+                                const int* n_frames_dev, int* status_dev, cudaStream_t s, int window_rows = 0);
+bool attention_scores_tc_supported(int dh);
 // partial[f][h][j] = sum_q exp(s(q,j) - lse[f][h][q]);  score[f][j] = sum_h partial / (heads*L)
 void launch_attention_scores_f32(const float* qkv, const float* lse, float* partial, float* score, int n_cap, int L,
                                  int heads, int dh, const int* n_frames_dev, cudaStream_t s);

@@ -140,12 +140,49 @@ __global__ void rope_pairs_kernel(T* __restrict__ qkv, const float2* __restrict_
   }
 }
 
+// The same, eight pairs per thread with 16-byte accesses (bf16 rows, dh/2 a multiple of 8).
+__global__ void rope_pairs_vec8_kernel(bf16* __restrict__ qkv, const float2* __restrict__ table, int rows_cap, int L,
+                                       int heads, int dh, const int* __restrict__ n_frames_dev) {
+  const int rows = n_frames_dev ? min(rows_cap, *n_frames_dev * L) : rows_cap;
+  const int half = dh >> 1, D = heads * dh, chunks = half >> 3;
+  const long long per_row = 2LL * heads * chunks;
+  const long long total = (long long)rows * per_row;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int r = (int)(idx / per_row);
+    int rem = (int)(idx % per_row);
+    const int which = rem / (heads * chunks);           // 0 = Q, 1 = K
+    rem %= heads * chunks;
+    const int h = rem / chunks, i0 = (rem % chunks) * 8;
+    bf16* p = qkv + (size_t)r * 3 * D + (size_t)which * D + h * dh + i0;
+    const float2* cs = table + (size_t)(r % L) * half + i0;
+    uint4 va = *reinterpret_cast<const uint4*>(p), vb = *reinterpret_cast<const uint4*>(p + half);
+    __nv_bfloat162* a2 = reinterpret_cast<__nv_bfloat162*>(&va);
+    __nv_bfloat162* b2 = reinterpret_cast<__nv_bfloat162*>(&vb);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 a = __bfloat1622float2(a2[j]), b = __bfloat1622float2(b2[j]);
+      const float2 c0 = __ldg(cs + 2 * j), c1 = __ldg(cs + 2 * j + 1);
+      a2[j] = __floats2bfloat162_rn(a.x * c0.x - b.x * c0.y, a.y * c1.x - b.y * c1.y);
+      b2[j] = __floats2bfloat162_rn(b.x * c0.x + a.x * c0.y, b.y * c1.x + a.y * c1.y);
+    }
+    *reinterpret_cast<uint4*>(p) = va;
+    *reinterpret_cast<uint4*>(p + half) = vb;
+  }
+}
+
 void launch_rope_pairs(void* qkv, const float2* table, int rows_cap, int L, int heads, int dh, bool is_bf16,
                        const int* n_frames_dev, cudaStream_t s) {
   if (rows_cap <= 0) return;
+  ET_COUNT_LAUNCH();
+  if (is_bf16 && (dh / 2) % 8 == 0 && (heads * dh) % 8 == 0) {
+    const long long total = (long long)rows_cap * heads * (dh / 8);
+    const int blocks = (int)min((total + 255) / 256, 148LL * 32);
+    rope_pairs_vec8_kernel<<<blocks, 256, 0, s>>>((bf16*)qkv, table, rows_cap, L, heads, dh, n_frames_dev);
+    return;
+  }
   const long long total = (long long)rows_cap * heads * dh;
   const int blocks = (int)min((total + 255) / 256, 148LL * 32);
-  ET_COUNT_LAUNCH();
   if (is_bf16) rope_pairs_kernel<bf16><<<blocks, 256, 0, s>>>((bf16*)qkv, table, rows_cap, L, heads, dh, n_frames_dev);
   else rope_pairs_kernel<float><<<blocks, 256, 0, s>>>((float*)qkv, table, rows_cap, L, heads, dh, n_frames_dev);
 }

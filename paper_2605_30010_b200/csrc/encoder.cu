@@ -19,10 +19,14 @@ void launch_score_finish(const float* partial, float* score, int n_cap, int L, i
 
 namespace {
 
-// dst[row(n)][k_pad] (bf16, zero padded for k >= K) = src[k][n] (fp32); row(n) = n for n < split, n + shift beyond
-// (the [gate | up] weight of a gated MLP is stored with each half padded to the same width)
+// Row of output j of a gated MLP ([gate | up]) in the order the fused epilogue of the dense layer wants: tiles of 256
+// rows = 128 outputs, inside a tile four groups of (32 gate rows, 32 up rows) of the same 32 outputs.
+__host__ __device__ inline int gated_row(int j, int up) { return (j >> 7) * 256 + ((j & 127) >> 5) * 64 + up * 32 + (j & 31); }
+
+// dst[row(n)][k_pad] (bf16, zero padded for k >= K) = src[k][n] (fp32); row(n) = n, or, with gated_M > 0 (source
+// columns [gate (gated_M) | up (gated_M)]), gated_row of the output (rows of padded outputs stay as they are)
 __global__ void transpose_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int K, int N, int k_pad,
-                                         int split, int shift) {
+                                         int gated_M) {
   __shared__ float tile[32][33];
   const int k0 = blockIdx.y * 32, n0 = blockIdx.x * 32;
   for (int i = threadIdx.y; i < 32; i += blockDim.y) {
@@ -32,7 +36,10 @@ __global__ void transpose_to_bf16_kernel(const float* __restrict__ src, bf16* __
   __syncthreads();
   for (int i = threadIdx.y; i < 32; i += blockDim.y) {
     const int n = n0 + i, k = k0 + threadIdx.x;
-    if (n < N && k < k_pad) dst[(size_t)(n < split ? n : n + shift) * k_pad + k] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+    if (n < N && k < k_pad) {
+      const int row = gated_M > 0 ? gated_row(n >= gated_M ? n - gated_M : n, n >= gated_M ? 1 : 0) : n;
+      dst[(size_t)row * k_pad + k] = __float2bfloat16_rn(tile[threadIdx.x][i]);
+    }
   }
 }
 
@@ -70,8 +77,7 @@ struct et_encoder {
   float* zeros = nullptr;                                   // [max(D, 2*Mp)] zero bias / zero position row
   float* bgu_pad = nullptr;                                 // [layers][2*Mp] gate | up biases in the padded layout (bf16 path)
   int* n_windows = nullptr;                                 // [1] attention windows alive = frames alive * wpf
-  void* GU = nullptr;                                       // [rows][2*Mp] gate | up pre-activations
-  TmaDesc c_GU;
+  void* GU = nullptr;                                       // fp32 path: [rows][2*M] gate | up pre-activations
   int device = 0;
   std::string last_error;
   std::vector<void*> dev_allocs, host_allocs;
@@ -90,7 +96,7 @@ struct et_encoder {
   TmaDesc d_Pm, d_Xn, d_O, d_Hm;                   // operand (A) maps
   TmaDesc c_X[2], c_QKV, c_Hm;                      // output (C) maps
   AttnMaps attn_maps;                               // QKV as seen by the tcgen05 attention kernel
-  bool attn_tc = false;
+  bool attn_tc = false, scores_tc = false;
   float *lse = nullptr, *score_partial = nullptr, *scores = nullptr, *simbuf = nullptr;
   float* frames_stage = nullptr;               // device staging for the *_host entry point (lazy)
 
@@ -213,7 +219,8 @@ et_status validate_config(const et_config* c) {
   if (c->hidden / c->heads > 128) return ET_ERR_SHAPE;
   if (c->mlp_dim < 1) return ET_ERR_SHAPE;
   if (c->dtype != ET_F32 && c->dtype != ET_BF16) return ET_ERR_INVALID_ARG;
-  if (c->dtype == ET_BF16 && (c->hidden % 8 != 0 || c->mlp_dim % 8 != 0 || (c->hidden / c->heads) % 8 != 0)) return ET_ERR_SHAPE;
+  // (the gated MLP of arch 1 is stored padded to a multiple of 64 columns, so its width is free)
+  if (c->dtype == ET_BF16 && (c->hidden % 8 != 0 || (c->arch != 1 && c->mlp_dim % 8 != 0) || (c->hidden / c->heads) % 8 != 0)) return ET_ERR_SHAPE;
   if (c->max_frames_total < 1 || c->max_videos < 1 || c->max_videos > 1024) return ET_ERR_INVALID_ARG;
   if (c->max_frames_total / (c->temporal_patch > 1 ? c->temporal_patch : 1) > 65535) return ET_ERR_CAPACITY;   // frames index gridDim.y
   if (c->arch == 1 && c->temporal_patch >= 1 && c->max_frames_total < c->temporal_patch) return ET_ERR_INVALID_ARG;
@@ -361,13 +368,14 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     const int a_cap = windowed ? T * e->wpf : T, a_L = windowed ? e->Lw : L;
     const int* a_n = windowed ? e->n_windows : n_dev;
     PROF(ET_CAT_ATTENTION, {
-      if (e->attn_tc) ET_CUDA(e, launch_attention_tc(e->attn_maps, (bf16*)e->O, e->lse, a_cap, a_L, H, dh, a_n, e->d_small + 10, s));
+      // the tensor-core kernel sweeps whole frames and masks the keys outside a query's window
+      if (e->attn_tc) ET_CUDA(e, launch_attention_tc(e->attn_maps, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, e->d_small + 10, s, windowed ? e->Lw : 0));
       else if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, a_cap, a_L, H, dh, a_n, s);
       else launch_attention_f32((const float*)e->QKV, (float*)e->O, e->lse, a_cap, a_L, H, dh, a_n, s);
     });
     if (layer == c.num_layers - 1) {
       PROF(ET_CAT_SCORES, {
-        if (e->attn_tc) ET_CUDA(e, launch_attention_scores_tc(e->attn_maps, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, e->d_small + 10, s));
+        if (e->scores_tc) ET_CUDA(e, launch_attention_scores_tc(e->attn_maps, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, e->d_small + 10, s));
         else if (e->bf) launch_attention_scores_bf16((const bf16*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
         else launch_attention_scores_f32((const float*)e->QKV, e->lse, e->score_partial, e->scores, T, L, H, dh, n_dev, s);
       });
@@ -378,9 +386,14 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     if (qw) {
       // gated MLP: [gate | up] pre-activations, silu(gate) * up, down projection added to the residual stream
       const int Mp = e->Mp;
-      PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, b ? b->d_w1 : none, e->c_GU, e->bf ? e->bgu_pad + (size_t)layer * 2 * Mp : W + o.b1,
-                   e->GU, rows_cap, 2 * Mp, D, EPI_STORE, nullptr, 1, n_dev, s)));
-      PROF(ET_CAT_GEMM, launch_gated_silu(e->GU, e->Hm, rows_cap, Mp, e->bf, n_dev, L, s));
+      if (e->bf) {
+        PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, nullptr, b->d_w1, e->c_Hm, e->bgu_pad + (size_t)layer * 2 * Mp, e->Hm, rows_cap,
+                     2 * Mp, D, EPI_SWIGLU, nullptr, 1, n_dev, s)));
+      } else {
+        PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Xn, e->d_Xn, W + o.w1, none, e->c_Hm, W + o.b1, e->GU, rows_cap, 2 * Mp, D, EPI_STORE, nullptr, 1,
+                     n_dev, s)));
+        PROF(ET_CAT_GEMM, launch_gated_silu(e->GU, e->Hm, rows_cap, Mp, false, n_dev, L, s));
+      }
       PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Hm, e->d_Hm, W + o.w2, b ? b->d_w2 : none, e->c_X[cur], W + o.b2, e->X[cur], rows_cap, D, Mp, EPI_RESIDUAL,
                    nullptr, 1, n_dev, s)));
     } else {
@@ -535,7 +548,7 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   e->ws = config->arch == 1 ? config->window : 0;
   e->wpf = e->ws > 0 ? (g / e->ws) * (g / e->ws) : 1;
   e->Lw = e->ws > 0 ? e->ws * e->ws : L;
-  e->Mp = (config->arch == 1 && e->bf) ? (config->mlp_dim + 63) / 64 * 64 : config->mlp_dim;
+  e->Mp = (config->arch == 1 && e->bf) ? (config->mlp_dim + 127) / 128 * 128 : config->mlp_dim;   // whole 128-output tiles
   e->Fmax = config->max_frames_total / tp; e->Vmax = config->max_videos;
   if (cudaGetDevice(&e->device) != cudaSuccess) return bail(ET_ERR_CUDA);
   const size_t D = config->hidden, M = config->mlp_dim, F = e->Fmax, rows = F * (size_t)L;
@@ -589,10 +602,9 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   ET_A(e->Pm, rows * e->Kp * es); ET_A(e->Xn, rows * D * es); ET_A(e->QKV, rows * 3 * D * es);
   ET_A(e->O, rows * D * es); ET_A(e->Hm, rows * Mp * es);
   if (e->arch == 1) {
-    ET_A(e->GU, rows * 2 * Mp * es);
+    if (!e->bf) ET_A(e->GU, rows * 2 * Mp * es);      // the tensor-core path applies the gate inside the dense layer
     ET_A(e->zeros, std::max(D, 2 * Mp) * 4);
     ET_A(e->n_windows, 4);
-    cudaMemset(e->GU, 0, rows * 2 * Mp * es);
     cudaMemset(e->zeros, 0, std::max(D, 2 * Mp) * 4);
     // rotary table and token orders.  Internal order = window-major (windows row-major over the grid, tokens
     // row-major inside a window), so that a window is a run of Lw consecutive rows; raster order otherwise.
@@ -659,14 +671,14 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
   if (e->bf) {
     // transposed bf16 copies of the dense weights ([out][in], K contiguous) + their tensor maps
     const char* err = nullptr;
-    // rows_out > N: the N source columns land in rows [0, split) and [split + shift, ...), the rest stays zero
-    auto convert = [&](size_t off, int K, int N, int k_pad, bf16** dst, int rows_out = 0, int split = 0, int shift = 0) -> et_status {
-      if (rows_out <= 0) { rows_out = N; split = N; shift = 0; }
+    // gated_M > 0: the [gate | up] weight of a gated MLP, rows_out >= N rows in the fused epilogue's order (the rest zero)
+    auto convert = [&](size_t off, int K, int N, int k_pad, bf16** dst, int rows_out = 0, int gated_M = 0) -> et_status {
+      if (rows_out <= 0) rows_out = N;
       et_status s2 = dalloc(e, dst, (size_t)rows_out * k_pad);
       if (s2 != ET_OK) return s2;
       if (rows_out != N && cudaMemset(*dst, 0, (size_t)rows_out * k_pad * sizeof(bf16)) != cudaSuccess) return ET_ERR_CUDA;
       ET_COUNT_LAUNCH();
-      transpose_to_bf16_kernel<<<dim3(cdiv(N, 32), cdiv(k_pad, 32)), dim3(32, 8)>>>(e->w_blob + off, *dst, K, N, k_pad, split, shift);
+      transpose_to_bf16_kernel<<<dim3(cdiv(N, 32), cdiv(k_pad, 32)), dim3(32, 8)>>>(e->w_blob + off, *dst, K, N, k_pad, gated_M);
       return cudaGetLastError() == cudaSuccess ? ET_OK : ET_ERR_CUDA;
     };
     if ((st = convert(e->off_patch_w, P, (int)D, e->Kp, &e->patch_w_t)) != ET_OK) return bail(st);
@@ -678,8 +690,8 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
       if ((st = convert(o.wqkv, (int)D, (int)(3 * D), (int)D, &b.wqkv_t)) != ET_OK) return bail(st);
       if ((st = convert(o.wo, (int)D, (int)D, (int)D, &b.wo_t)) != ET_OK) return bail(st);
       if (e->arch == 1) {
-        // [gate | up]: 2M source columns -> 2*Mp rows, each half padded to Mp; down: K padded to Mp
-        if ((st = convert(o.w1, (int)D, (int)(2 * M), (int)D, &b.w1_t, (int)(2 * Mp), (int)M, (int)(Mp - M))) != ET_OK) return bail(st);
+        // [gate | up]: 2M source columns -> 2*Mp rows in the fused epilogue's order; down: K padded to Mp
+        if ((st = convert(o.w1, (int)D, (int)(2 * M), (int)D, &b.w1_t, (int)(2 * Mp), (int)M)) != ET_OK) return bail(st);
         if ((st = convert(o.w2, (int)M, (int)D, (int)Mp, &b.w2_t)) != ET_OK) return bail(st);
       } else {
         if ((st = convert(o.w1, (int)D, (int)M, (int)D, &b.w1_t)) != ET_OK) return bail(st);
@@ -695,16 +707,14 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
               make_tma_2d_bf16(&e->d_O, e->O, rows, D, 128, &err) && make_tma_2d_bf16(&e->d_Hm, e->Hm, rows, Mp, 128, &err) &&
               make_tma_out(&e->c_X[0], e->X[0], rows, D, true, &err) && make_tma_out(&e->c_X[1], e->X[1], rows, D, true, &err) &&
               make_tma_out(&e->c_QKV, e->QKV, rows, 3 * D, false, &err) && make_tma_out(&e->c_Hm, e->Hm, rows, Mp, false, &err);
-    if (ok && e->arch == 1) ok = make_tma_out(&e->c_GU, e->GU, rows, 2 * Mp, false, &err);
     if (!ok) return bail(fail(e, ET_ERR_CUDA, err ? err : "tensor map"));
     if (e->arch == 1) {
-      // gate | up biases in the padded layout
+      // gate | up biases in the order of the weight rows
       std::vector<float> hb((size_t)config->num_layers * 2 * Mp, 0.f);
       for (int i = 0; i < config->num_layers; ++i) {
         const float* src = weights->data + e->lo[i].b1;
         float* dst = hb.data() + (size_t)i * 2 * Mp;
-        memcpy(dst, src, M * sizeof(float));
-        memcpy(dst + Mp, src + M, M * sizeof(float));
+        for (size_t j = 0; j < M; ++j) { dst[gated_row((int)j, 0)] = src[j]; dst[gated_row((int)j, 1)] = src[M + j]; }
       }
       if ((st = dalloc(e, &e->bgu_pad, hb.size())) != ET_OK) return bail(st);
       if (cudaMemcpy(e->bgu_pad, hb.data(), hb.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) return bail(ET_ERR_CUDA);
@@ -713,6 +723,7 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
       if (!make_attention_maps(&e->attn_maps, (const bf16*)e->QKV, (long long)rows, config->heads, e->dh))
         return bail(fail(e, ET_ERR_CUDA, "tensor map of the attention operands"));
       e->attn_tc = true;
+      e->scores_tc = attention_scores_tc_supported(e->dh);
     }
   }
   if (cudaDeviceSynchronize() != cudaSuccess) return bail(ET_ERR_CUDA);
@@ -941,6 +952,31 @@ et_status et_attention(const void* qkv_dev, void* out_dev, float* lse_dev, int n
   return ET_OK;
 }
 
+et_status et_attention_windowed(const void* qkv_dev, void* out_dev, float* lse_scratch_dev, int n, int L, int heads,
+                                int head_dim, int window_rows, int dtype, void* cuda_stream) {
+  if (!qkv_dev || !out_dev || !lse_scratch_dev) return ET_ERR_INVALID_ARG;
+  if (n < 1 || L < 1 || heads < 1 || heads > 65535 || head_dim < 1 || head_dim > 128) return ET_ERR_SHAPE;
+  if (window_rows < 1 || L % window_rows != 0 || (long long)n * (L / window_rows) > 65535) return ET_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int items = n * (L / window_rows);
+  if (dtype == ET_BF16) {
+    if (head_dim % 8 != 0) return ET_ERR_SHAPE;
+    if (attention_tc_supported(head_dim)) {
+      AttnMaps maps;
+      if (!make_attention_maps(&maps, (const bf16*)qkv_dev, (long long)n * L, heads, head_dim)) return ET_ERR_CUDA;
+      ET_CUDA0(launch_attention_tc(maps, (bf16*)out_dev, lse_scratch_dev, n, L, heads, head_dim, nullptr, nullptr, s, window_rows));
+      return ET_OK;
+    }
+    launch_attention_bf16((const bf16*)qkv_dev, (bf16*)out_dev, lse_scratch_dev, items, window_rows, heads, head_dim, nullptr, s);
+  } else if (dtype == ET_F32) {
+    launch_attention_f32((const float*)qkv_dev, (float*)out_dev, lse_scratch_dev, items, window_rows, heads, head_dim, nullptr, s);
+  } else {
+    return ET_ERR_INVALID_ARG;
+  }
+  ET_CUDA0(cudaGetLastError());
+  return ET_OK;
+}
+
 et_status et_attention_scores(const void* qkv_dev, const float* lse_dev, float* partial_dev, float* score_dev, int n, int L,
                               int heads, int head_dim, int dtype, void* cuda_stream) {
   if (!qkv_dev || !lse_dev || !partial_dev || !score_dev) return ET_ERR_INVALID_ARG;
@@ -948,7 +984,7 @@ et_status et_attention_scores(const void* qkv_dev, const float* lse_dev, float* 
   cudaStream_t s = (cudaStream_t)cuda_stream;
   if (dtype == ET_BF16) {
     if (head_dim % 8 != 0) return ET_ERR_SHAPE;
-    if (attention_tc_supported(head_dim)) {
+    if (attention_scores_tc_supported(head_dim)) {
       AttnMaps maps;
       if (!make_attention_maps(&maps, (const bf16*)qkv_dev, (long long)n * L, heads, head_dim)) return ET_ERR_CUDA;
       ET_CUDA0(launch_attention_scores_tc(maps, lse_dev, partial_dev, score_dev, n, L, heads, head_dim, nullptr, nullptr, s));

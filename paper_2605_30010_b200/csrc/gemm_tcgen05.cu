@@ -305,7 +305,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
           if (n0 + c_first < g.N) tmem_ld32_async(t_row + (uint32_t)c_first, rr[0]);
           if constexpr (EPI == EPI_SWIGLU) {
             // Chunks come in pairs (gate, up) of the same 32 outputs (the weight rows were interleaved that way):
-            // h = silu(gate) * up, half as many output columns as accumulator columns.  No bias.
+            // h = silu(gate + b) * (up + b), half as many output columns as accumulator columns; the bias is in
+            // weight-row order.
             float gate[32];
 #pragma unroll
             for (int ch = 0; ch < CH_PER; ++ch) {
@@ -314,13 +315,17 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
               tmem_regs_ready(rr[ch & 1]);
               if (ch + 1 < CH_PER) tmem_ld32_async(t_row + (uint32_t)(c0 + 32), rr[(ch + 1) & 1]);
               const uint32_t (&r)[32] = rr[ch & 1];
+              float4 b[8];                              // bias of this chunk (weight-row order; zeros where a layer has none)
+#pragma unroll
+              for (int q = 0; q < 8; ++q) b[q] = __ldg(reinterpret_cast<const float4*>(g.bias + n0 + c0 + q * 4));
+              const float* bf = reinterpret_cast<const float*>(b);
               if ((ch & 1) == 0) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) gate[i] = __uint_as_float(r[i]);
+                for (int i = 0; i < 32; ++i) gate[i] = __uint_as_float(r[i]) + bf[i];
               } else {
                 float v[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = __fdividef(gate[i], 1.f + __expf(-gate[i])) * __uint_as_float(r[i]);
+                for (int i = 0; i < 32; ++i) v[i] = __fdividef(gate[i], 1.f + __expf(-gate[i])) * (__uint_as_float(r[i]) + bf[i]);
                 if (lane == 0) bulk_wait_read<1>();   // the half written two stores ago has been read
                 __syncwarp();
                 const uint32_t buf = slab + sub * 2048u;
@@ -415,8 +420,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constan
               float v[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                const float gt = __uint_as_float(rg[q * 8 + i]);
-                v[i] = __fdividef(gt, 1.f + __expf(-gt)) * __uint_as_float(ru[q * 8 + i]);
+                const float gt = __uint_as_float(rg[q * 8 + i]) + __ldg(g.bias + n0 + c0 + q * 8 + i);
+                v[i] = __fdividef(gt, 1.f + __expf(-gt)) * (__uint_as_float(ru[q * 8 + i]) + __ldg(g.bias + n0 + c0 + 32 + q * 8 + i));
               }
               uint4 o;
               o.x = pack_bf16(v[0], v[1]); o.y = pack_bf16(v[2], v[3]);

@@ -212,6 +212,8 @@ cudaError_t run(const AttnMaps& maps, const ScoreArgs& a, cudaStream_t s) {
 
 }  // namespace
 
+bool attention_scores_tc_supported(int dh) { return dh == 64 || dh == 72; }
+
 cudaError_t launch_attention_scores_tc(const AttnMaps& maps, const float* lse, float* partial, float* score, int n_cap,
                                        int L, int heads, int dh, const int* n_frames_dev, int* status_dev, cudaStream_t s) {
   if (n_cap <= 0) return cudaSuccess;

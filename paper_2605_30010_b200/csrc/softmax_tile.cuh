@@ -13,13 +13,13 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// maximum of the (valid) logits of one 32-column chunk whose first column is c0
+// maximum of the valid logits (columns lo <= c < nk of the tile) of one 32-column chunk whose first column is c0
 template <bool MASK>
-__device__ __forceinline__ float row_max(const uint32_t (&r)[32], int c0, int nk) {
+__device__ __forceinline__ float row_max(const uint32_t (&r)[32], int c0, int nk, int lo = 0) {
   float a[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
   for (int i = 0; i < 32; ++i)
-    if (!MASK || c0 + i < nk) a[i & 3] = fmaxf(a[i & 3], __uint_as_float(r[i]));
+    if (!MASK || (c0 + i < nk && c0 + i >= lo)) a[i & 3] = fmaxf(a[i & 3], __uint_as_float(r[i]));
   return fmaxf(fmaxf(a[0], a[1]), fmaxf(a[2], a[3]));
 }
 
@@ -27,7 +27,7 @@ __device__ __forceinline__ float row_max(const uint32_t (&r)[32], int c0, int nk
 // and ADD count, worth 4 % of the kernel; a three-input maximum and a cubic exp2 on the FMA pipe were measured slower.
 template <bool MASK>
 __device__ __forceinline__ void probs(const uint32_t (&r)[32], int c0, int nk, float scale2, float m, float (&ls)[4],
-                                      uint32_t p_addr) {
+                                      uint32_t p_addr, int lo = 0) {
   uint32_t pk[16];
   const float neg_m = -m;
 #pragma unroll
@@ -36,8 +36,8 @@ __device__ __forceinline__ void probs(const uint32_t (&r)[32], int c0, int nk, f
     fma2(x0, x1, __uint_as_float(r[i]), __uint_as_float(r[i + 1]), scale2, scale2, neg_m, neg_m);
     float p0 = ex2(x0), p1 = ex2(x1);
     if (MASK) {
-      if (c0 + i >= nk) p0 = 0.f;
-      if (c0 + i + 1 >= nk) p1 = 0.f;
+      if (c0 + i >= nk || c0 + i < lo) p0 = 0.f;
+      if (c0 + i + 1 >= nk || c0 + i + 1 < lo) p1 = 0.f;
     }
     const int a = ((i >> 1) & 1) * 2;                // two pairs of partial sums, alternating
     add2(ls[a], ls[a + 1], ls[a], ls[a + 1], p0, p1);

@@ -36,7 +36,8 @@ from oracle import earlytom_oracle as O  # noqa: E402
 from synthetic import make_batch, make_weights, workload  # noqa: E402
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-FULL_SIZE = ("so400m_32f", "so400m_32f_cal", "so400m_64f_p10", "so400m_64f_p50", "so400m_64f_p90", "serve_8x32")
+FULL_SIZE = ("so400m_32f", "so400m_32f_cal", "so400m_64f_p10", "so400m_64f_p50", "so400m_64f_p90", "serve_8x32",
+             "qwenvl_768f")
 ROW_STRIDE = 97
 
 

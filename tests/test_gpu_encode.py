@@ -250,6 +250,12 @@ def test_qwenvl_small_bf16(B):
     run_workload(B, wl, np.float64, BF16_TOL, BF16_SIM, BF16_SCORE)
 
 
+def test_qwenvl_32f_bf16(B):
+    """Qwen2.5-VL's own widths (1280, 16 heads of 80, gated MLP 3420, 32 blocks, windows of 64 tokens in frames of 256):
+    16 encoder frames; the oracle runs in the test (about half a minute)."""
+    run_workload(B, workload("qwenvl_32f"), np.float32, BF16_TOL, BF16_SIM, BF16_SCORE)
+
+
 def test_qwenvl_argument_errors(B):
     wl = workload("qwenvl_tiny")
     frames, offs = make_batch(wl)

@@ -282,7 +282,7 @@ def test_attention_f32(B, n, L, H, dh):
 @pytest.mark.parametrize("n,L,H,dh", [(2, 729, 16, 72), (1, 64, 4, 16), (1, 100, 2, 64), (3, 130, 2, 72),
                                       (1, 17, 1, 32), (1, 200, 1, 128), (1, 70, 2, 40),
                                       (2, 128, 1, 72), (1, 257, 2, 72), (3, 1, 1, 72), (5, 16, 3, 64), (1, 513, 1, 72),
-                                      (40, 729, 2, 72)])
+                                      (40, 729, 2, 72), (2, 256, 4, 80), (1, 729, 2, 80), (3, 64, 2, 80), (2, 300, 1, 80)])
 def test_attention_bf16(B, n, L, H, dh):
     import torch
     rng = np.random.default_rng(L + dh)
@@ -296,6 +296,24 @@ def test_attention_bf16(B, n, L, H, dh):
     np.testing.assert_allclose(score * L, score_ref * L, rtol=1e-3, atol=1e-4)
     s2 = B.et_attention_scores(qkv.cuda(), lse, n, L, H, dh).cpu().numpy()
     assert (s2 == score).all(), "score pass must be bit-reproducible"
+
+
+@pytest.mark.parametrize("n,L,H,dh,w,bf", [(2, 256, 2, 80, 64, True), (3, 64, 2, 80, 16, True), (1, 512, 1, 72, 128, True),
+                                          (2, 384, 2, 64, 96, True), (1, 256, 1, 80, 256, True), (2, 36, 3, 16, 9, False),
+                                          (1, 320, 2, 40, 64, True)])
+def test_attention_windowed(B, n, L, H, dh, w, bf):
+    """Windows are runs of w consecutive rows: the result equals plain attention over each window on its own."""
+    rng = np.random.default_rng(L + dh + w)
+    qkv = rng.standard_normal((n * L, 3 * H * dh)).astype(np.float32)
+    if bf:
+        qkv = bf16_round(qkv)
+        out = B.et_attention_windowed(qkv.cuda(), n, L, H, dh, w).float().cpu().numpy()
+        ref, _, _ = attention_ref(qkv.float().numpy(), n * (L // w), w, H, dh)
+        assert np.abs(out - ref).max() <= 2e-2 * np.abs(ref).max()
+    else:
+        out = B.et_attention_windowed(cuda(qkv), n, L, H, dh, w).cpu().numpy()
+        ref, _, _ = attention_ref(qkv, n * (L // w), w, H, dh)
+        np.testing.assert_allclose(out, ref, rtol=0, atol=2e-5)
 
 
 @pytest.mark.parametrize("rows,D,bf", [(100, 64, False), (333, 1152, True), (5, 2048, False), (17, 12, True)])

@@ -81,7 +81,8 @@ def test_swiglu(B, rows, M):
 
 @pytest.mark.parametrize("rows,K,M", [(300, 256, 128), (1000, 512, 1408), (77, 64, 256)])
 def test_gated_dense_layer(B, rows, K, M):
-    """Dense layer with the SwiGLU epilogue: weight rows in the interleaved order, output silu(gate) * up."""
+    """Dense layer with the SwiGLU epilogue: weight rows and bias in the interleaved order, output
+    silu(gate + b_gate) * (up + b_up)."""
     import torch
     rng = np.random.default_rng(K + M)
     a, a_ref = _bf16(rng.standard_normal((rows, K)))
@@ -92,10 +93,13 @@ def test_gated_dense_layer(B, rows, K, M):
     w = torch.empty((2 * M, K), dtype=torch.bfloat16, device="cuda")
     w[torch.from_numpy(row_gate).cuda()] = wg
     w[torch.from_numpy(row_gate + 32).cuda()] = wu
+    bg, bu = (0.3 * rng.standard_normal(M)).astype(np.float32), (0.3 * rng.standard_normal(M)).astype(np.float32)
     bias = torch.zeros(2 * M, dtype=torch.float32, device="cuda")
+    bias[torch.from_numpy(row_gate).cuda()] = torch.from_numpy(bg).cuda()
+    bias[torch.from_numpy(row_gate + 32).cuda()] = torch.from_numpy(bu).cuda()
     h, status = B.et_linear_bf16(a, w, bias, epilogue=4)
     assert int(status.item()) == 0 and tuple(h.shape) == (rows, M)
-    ref = P.silu(a_ref @ wg_ref.T) * (a_ref @ wu_ref.T)
+    ref = P.silu(a_ref @ wg_ref.T + bg) * (a_ref @ wu_ref.T + bu)
     got = h.float().cpu().numpy().astype(np.float64)
     assert np.abs(got - ref).max() <= 1.5 * BF16_ULP * np.abs(ref).max() + 1e-5, f"error {np.abs(got - ref).max():.3e}"
     err = np.abs(got - ref)
