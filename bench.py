@@ -117,7 +117,7 @@ def oracle_sample(wl, frames, blob, sample_frames, steps, warmup):
     w = O.split_weights(wl.shape, blob)
     sub = frames[:sample_frames]
     for _ in range(warmup):
-        O.encode_video(sub[:1], wl.shape, w, wl.params, dtype=np.float32)
+        O.encode_video(sub[:wl.shape.temporal_patch], wl.shape, w, wl.params, dtype=np.float32)
     t0 = time.perf_counter()
     for _ in range(steps):
         r = O.encode_video(sub, wl.shape, w, wl.params, dtype=np.float32)
@@ -130,11 +130,12 @@ def oracle_sample(wl, frames, blob, sample_frames, steps, warmup):
     return sample_frames / dt, dt, cores, len(r.frame_dynamic), int(r.tokens.shape[0])
 
 
-def sample_note(sample, total, frames_out, tokens_out, L):
-    merged = "no merge executed: Stage I needs four frames in a segment" if sample < 4 else \
-        f"Stage I left {frames_out} of {sample} frames"
+def sample_note(sample, total, frames_out, tokens_out, L, tp=1):
+    enc = sample // tp                  # encoder frames (tp input frames each)
+    merged = "no merge executed: Stage I needs four frames in a segment" if enc < 4 else \
+        f"Stage I left {frames_out} of {enc} encoder frames"
     return (f"first {sample} of {total} frames of the same video, numpy fp32 oracle, whole method ({merged}; "
-            f"{tokens_out} of {sample * L} tokens kept)")
+            f"{tokens_out} of {enc * L} tokens kept)")
 
 
 def run_reference(args, wl):
@@ -147,9 +148,10 @@ def run_reference(args, wl):
     # The oracle needs 6-10 s per frame on 8-16 host cores.  The sample per step is sized so that the whole
     # --steps K run stays near three minutes: 8 frames per step (Stage I merges) up to K = 3, one frame at K = 20.
     steps = max(1, args.steps)
-    sample = int(max(1, min(8, wl.videos[0].n_frames, 24 // steps)))
+    tp = wl.shape.temporal_patch
+    sample = int(max(1, min(8, wl.videos[0].n_frames // tp, 24 // steps))) * tp
     fps, dt, cores, n_out, t_out = oracle_sample(wl, frames, blob, sample, steps, min(1, args.warmup))
-    note = sample_note(sample, wl.total_frames, n_out, t_out, wl.shape.tokens_per_frame)
+    note = sample_note(sample, wl.total_frames, n_out, t_out, wl.shape.tokens_per_frame, tp)
     line = {"impl": "reference", "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -580,10 +582,10 @@ def main():
         except Exception as ex:
             line["hbm_kernels"] = {"error": f"{type(ex).__name__}: {ex}"[:300]}
     if not args.no_cpu_baseline:
-        sample = min(8, wl.videos[0].n_frames)
+        sample = min(8 * shape.temporal_patch, wl.videos[0].n_frames)
         fps, dt, cores, n_out, t_out = oracle_sample(wl, vids[0], blob, sample, 1, 1)
         line["cpu_baseline"] = {"value": fps, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": sample_note(sample, T, n_out, t_out, shape.tokens_per_frame) + f", {dt:.1f} s"}
+                                "sample": sample_note(sample, T, n_out, t_out, shape.tokens_per_frame, shape.temporal_patch) + f", {dt:.1f} s"}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

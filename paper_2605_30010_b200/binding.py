@@ -24,7 +24,7 @@ EXPORTS = ["et_encoder_create", "et_encode_video", "et_encode_batch", "et_encode
            "et_status_string", "et_last_error", "et_kernel_launch_count", "et_profile_enable", "et_profile_read",
            "et_selftest_bounded_wait", "et_debug_build", "et_debug_status",
            "et_frame_similarity_static", "et_frame_similarity", "et_merge_plan",
-           "et_merge_frames", "et_select_tokens", "et_gather_tokens", "et_linear_bf16", "et_attention",
+           "et_merge_frames", "et_select_tokens", "et_gather_tokens", "et_linear_bf16", "et_attention", "et_attention_windowed",
            "et_attention_scores", "et_layernorm",
            # include/earlytom_llm.h
            "et_llm_create", "et_llm_prefill", "et_llm_destroy", "et_llm_last_error", "et_llm_profile_enable",

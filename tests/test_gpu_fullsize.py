@@ -33,7 +33,7 @@ pytestmark = pytest.mark.gpu
 BF16_TOL = 2e-2
 BF16_SIM, BF16_SCORE = 5e-4, 1e-2     # hard ceilings on similarity / score error (see tests/test_gpu_encode.py)
 NEAR_TIE_SHARE = 0.005
-FULL_SIZE = ["so400m_32f", "so400m_32f_cal", "so400m_64f_p50", "so400m_64f_p10", "so400m_64f_p90", "serve_8x32"]
+FULL_SIZE = ["so400m_32f", "so400m_32f_cal", "so400m_64f_p50", "so400m_64f_p10", "so400m_64f_p90", "serve_8x32", "qwenvl_768f"]
 
 
 @pytest.fixture(scope="module")
@@ -89,7 +89,7 @@ def _check_decisions(run, wl, offs):
     # Stage II amounts and kept sets
     for v in range(len(cur) - 1):
         f0, f1 = int(cur[v]), int(cur[v + 1])
-        Bv = int(offs[v + 1] - offs[v])
+        Bv = int(offs[v + 1] - offs[v])                  # encoder frames of the video
         k, w, M = O.rescaled_keep(p.retain, Bv, f1 - f0, L, p.retain_mode, p.window_mode)
         assert tr.video_k[v] == k and tr.video_w[v] == w
         keep = O.select_tokens(tr.scores[f0:f1].astype(np.float64), run["dynamic"][f0:f1], k, w, p.selection, p.window_mode)
@@ -132,7 +132,7 @@ def test_full_size_against_oracle(B, name):
     assert stats["near_ties"] <= max(1, NEAR_TIE_SHARE * stats["decisions"]), stats
     # the budget of Eq. 5: with k near-equal windows on static frames the kept total is N*k per video
     L = wl.shape.tokens_per_frame
-    target = wl.params.retain * wl.total_frames * L
+    target = wl.params.retain * wl.encoder_frames * L
     assert abs(ob.n_tokens - target) <= len(ob.dynamic), (ob.n_tokens, target)
 
 
@@ -140,35 +140,38 @@ def test_full_size_against_oracle(B, name):
 def test_full_size_workload(B, name):
     import torch
     wl = workload(name)
-    shape, L = wl.shape, wl.shape.tokens_per_frame
-    frames, offs = make_batch(wl)
+    shape, L, tp = wl.shape, wl.shape.tokens_per_frame, wl.shape.temporal_patch
+    frames, in_offs = make_batch(wl)
+    offs = [int(o) // tp for o in in_offs]              # every index the library reports is in encoder frames
     blob = make_weights(shape, wl.weight_seed, wl.pos_std)
     enc = B.Encoder(shape, blob, B.ET_BF16, wl.total_frames, len(wl.videos))
     try:
         fr = torch.from_numpy(frames).cuda()
-        unc = _snapshot(enc.encode_batch(fr, offs, wl.uncompressed().params))
-        run = _snapshot(enc.encode_batch(fr, offs, wl.params, want_trace=True))
-        again = _snapshot(enc.encode_batch(fr, offs, wl.params))
+        unc = _snapshot(enc.encode_batch(fr, in_offs, wl.uncompressed().params))
+        run = _snapshot(enc.encode_batch(fr, in_offs, wl.params, want_trace=True))
+        again = _snapshot(enc.encode_batch(fr, in_offs, wl.params))
     finally:
         enc.close()
-    assert unc["n_tokens"] == wl.total_frames * L
+    assert unc["n_tokens"] == wl.encoder_frames * L
     assert np.array_equal(run["tokens"], again["tokens"]) and np.array_equal(run["token_pos"], again["token_pos"]), \
         "two runs of the same call must agree bit for bit"
 
     # values: sampled frames of the uncompressed run against the oracle on those frames alone
     w = O.split_weights(shape, blob)
-    samples = [0, wl.total_frames - 1] if name in ("so400m_32f", "serve_8x32") else [wl.total_frames // 2]
+    samples = [0, wl.encoder_frames - 1] if name in ("so400m_32f", "serve_8x32") else [wl.encoder_frames // 2]
     if name == "so400m_32f_cal":
         samples = [6]                       # the first scene cut
+    if name == "qwenvl_768f":
+        samples = [0, 24, 383]              # first frame, a scene cut, last frame
     for fidx in samples:
-        ref = O.encode_video(frames[fidx:fidx + 1], shape, w, wl.uncompressed().params, dtype=np.float32)
+        ref = O.encode_video(frames[fidx * tp:(fidx + 1) * tp], shape, w, wl.uncompressed().params, dtype=np.float32)
         err = H.token_error(unc["tokens"][fidx * L:(fidx + 1) * L], ref.tokens)
         assert err <= BF16_TOL, f"{name} frame {fidx}: token error {err:.3e}"
 
     # decisions and structure
     _check_decisions(run, wl, offs)
     _check_structure(run, offs, L)
-    expect_blocks, alive, m = [], wl.total_frames, 0
+    expect_blocks, alive, m = [], wl.encoder_frames, 0
     for layer in range(shape.num_layers):
         if m < len(wl.params.merge_layers) and wl.params.merge_layers[m] == layer:
             alive = run["trace"].n_out[m]; m += 1
@@ -187,5 +190,5 @@ def test_full_size_workload(B, name):
             assert np.array_equal(run["tokens"][a:b], unc["tokens"][rows]), f"{name}: un-merged frame {f} differs"
             checked += 1
     assert checked > 0
-    retained = run["n_tokens"] / (wl.total_frames * L)
-    print(f"{name}: frames {wl.total_frames} -> {run['n_frames']}, tokens kept {retained:.3f}, un-merged frames checked {checked}")
+    retained = run["n_tokens"] / (wl.encoder_frames * L)
+    print(f"{name}: frames {wl.encoder_frames} -> {run['n_frames']}, tokens kept {retained:.3f}, un-merged frames checked {checked}")
