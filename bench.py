@@ -29,7 +29,7 @@ sys.path.insert(0, ROOT)
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of gemm_bf16_kernel<256, *>, average of the four dense
 # launches of block 0 at 32 frames (one ncu capture of this workload).  Re-taken whenever that kernel changes.
-GEMM_DRAM_BYTES_PER_LAUNCH = 251.0e6
+GEMM_DRAM_BYTES_PER_LAUNCH = 251.5e6
 
 METRIC = "frames/s through compressed encoder (32f SigLIP-so400m)"
 UNIT = "frames/s"
