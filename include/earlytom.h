@@ -200,6 +200,31 @@ ET_API et_status et_encode_batch_host(et_encoder* enc, const float* frames_host,
                                const et_params* params, void* cuda_stream, const et_host_buffers* dst,
                                et_result* out);
 
+/* The same host-to-host call split in two, so that the copies of neighbouring calls overlap the
+ * encoder's work (no counterpart in the paper: serving plumbing around Fig. 3's pipeline).
+ *
+ * et_encode_batch_host_submit validates like et_encode_batch_host, enqueues the upload of
+ * frames_host on a copy stream of the encoder's own and every kernel of the call on cuda_stream
+ * behind it, and returns without waiting; *ticket names the call.  At most TWO calls may be in
+ * flight (ET_ERR_CAPACITY on a third); each owns its own frame staging area and result buffers,
+ * while the work buffers are shared, so calls in flight together must name the same cuda_stream
+ * (ET_ERR_INVALID_ARG otherwise) and run one after the other on the device.  frames_host and the
+ * buffers of dst stay the caller's and must remain valid and untouched until the call is collected;
+ * pinned memory is needed for the upload to overlap.  params and video_offsets_host are copied.
+ * params->forced_plan, params->want_trace and et_profile_enable need the synchronous calls
+ * (ET_ERR_INVALID_ARG).  The synchronous encode calls are refused while a call is in flight.
+ *
+ * et_encode_batch_host_collect waits for that call's kernels, reads its status and sizes, copies
+ * tokens and index map into the dst given at submit (ET_ERR_CAPACITY if too small), waits for those
+ * copies and fills *out; out's device pointers name the call's slot and stay valid until the second
+ * next submit or the next synchronous call.  Calls are collected in submission order (ET_ERR_INVALID_ARG otherwise, and for a
+ * ticket that is not in flight).  A call that fails at collect is over: its slot is free again.
+ * Results are bit-identical to et_encode_batch_host's on the same inputs. */
+ET_API et_status et_encode_batch_host_submit(et_encoder* enc, const float* frames_host, const int* video_offsets_host,
+                                      int V, const et_params* params, void* cuda_stream,
+                                      const et_host_buffers* dst, unsigned long long* ticket);
+ET_API et_status et_encode_batch_host_collect(et_encoder* enc, unsigned long long ticket, et_result* out);
+
 ET_API void et_destroy(et_encoder* enc);
 ET_API const char* et_status_string(et_status s);
 ET_API const char* et_last_error(const et_encoder* enc); /* text of the last failure on this encoder */

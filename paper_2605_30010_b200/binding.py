@@ -20,7 +20,8 @@ ET_F32, ET_BF16 = 0, 1
 ET_MAX_MERGE_LAYERS = 8
 STATUS_NAMES = ["ET_OK", "ET_ERR_INVALID_ARG", "ET_ERR_SHAPE", "ET_ERR_CAPACITY", "ET_ERR_OOM", "ET_ERR_CUDA",
                 "ET_ERR_TIMEOUT", "ET_ERR_WEIGHTS"]
-EXPORTS = ["et_encoder_create", "et_encode_video", "et_encode_batch", "et_encode_batch_host", "et_destroy",
+EXPORTS = ["et_encoder_create", "et_encode_video", "et_encode_batch", "et_encode_batch_host", "et_encode_batch_host_submit",
+           "et_encode_batch_host_collect", "et_destroy",
            "et_status_string", "et_last_error", "et_kernel_launch_count", "et_profile_enable", "et_profile_read",
            "et_selftest_bounded_wait", "et_debug_build", "et_debug_status",
            "et_frame_similarity_static", "et_frame_similarity", "et_merge_plan",
@@ -136,6 +137,9 @@ def load_library(path: str = _LIB_PATH) -> C.CDLL:
     lib.et_encode_batch.argtypes = [vp, vp, _I32P, i, C.POINTER(et_params), vp, C.POINTER(et_result)]
     lib.et_encode_batch_host.argtypes = [vp, vp, _I32P, i, C.POINTER(et_params), vp, C.POINTER(et_host_buffers),
                                          C.POINTER(et_result)]
+    lib.et_encode_batch_host_submit.argtypes = [vp, vp, _I32P, i, C.POINTER(et_params), vp, C.POINTER(et_host_buffers),
+                                                C.POINTER(C.c_ulonglong)]
+    lib.et_encode_batch_host_collect.argtypes = [vp, C.c_ulonglong, C.POINTER(et_result)]
     lib.et_destroy.argtypes = [vp]
     lib.et_destroy.restype = None
     lib.et_status_string.argtypes = [i]
@@ -420,6 +424,15 @@ class HostBuffers:
                                  capacity_tokens, capacity_frames)
 
 
+def _host_result(enc: Encoder, r, dst: HostBuffers) -> Result:
+    N, nt, V = r.n_frames_out, r.n_tokens, r.n_videos
+    return Result(n_videos=V, n_frames_in=r.n_frames_in, n_frames_out=N, n_tokens=nt, tokens=dst.tokens[:nt],
+                  video_frame_offsets=dst.video_frame_offsets[:V + 1], frame_offsets=dst.frame_offsets[:N + 1],
+                  frame_src_lo=dst.frame_src_lo[:N], frame_src_hi=dst.frame_src_hi[:N],
+                  frame_dynamic=dst.frame_dynamic[:N], token_pos=dst.token_pos[:nt],
+                  frames_per_block=[r.frames_per_block[i] for i in range(enc.num_layers)])
+
+
 def et_encode_batch_host(enc: Encoder, frames_host, video_offsets: Sequence[int], params, dst: HostBuffers,
                          stream=None) -> Result:
     """frames_host: CPU torch tensor (pinned for asynchronous copies) [T,3,H,W] float32."""
@@ -429,12 +442,33 @@ def et_encode_batch_host(enc: Encoder, frames_host, video_offsets: Sequence[int]
     r = et_result()
     _check(lib().et_encode_batch_host(enc.handle, _ptr(frames_host), offs.ctypes.data_as(_I32P), len(offs) - 1,
                                       C.byref(q), _stream_ptr(stream), C.byref(dst.c), C.byref(r)), enc.handle)
-    N, nt, V = r.n_frames_out, r.n_tokens, r.n_videos
-    return Result(n_videos=V, n_frames_in=r.n_frames_in, n_frames_out=N, n_tokens=nt, tokens=dst.tokens[:nt],
-                  video_frame_offsets=dst.video_frame_offsets[:V + 1], frame_offsets=dst.frame_offsets[:N + 1],
-                  frame_src_lo=dst.frame_src_lo[:N], frame_src_hi=dst.frame_src_hi[:N],
-                  frame_dynamic=dst.frame_dynamic[:N], token_pos=dst.token_pos[:nt],
-                  frames_per_block=[r.frames_per_block[i] for i in range(enc.num_layers)])
+    return _host_result(enc, r, dst)
+
+
+class HostCall:
+    """A submitted host call: the ticket plus references that keep its host buffers alive until it is collected."""
+
+    def __init__(self, ticket: int, frames_host, dst: HostBuffers):
+        self.ticket, self.frames_host, self.dst = ticket, frames_host, dst
+
+
+def et_encode_batch_host_submit(enc: Encoder, frames_host, video_offsets: Sequence[int], params, dst: HostBuffers,
+                                stream=None) -> HostCall:
+    """Enqueues upload and encode and returns at once; at most two calls in flight, collected in order."""
+    assert not frames_host.is_cuda and frames_host.is_contiguous()
+    offs = np.ascontiguousarray(np.asarray(video_offsets, dtype=np.int32))
+    q, keep = make_params(params)
+    ticket = C.c_ulonglong(0)
+    _check(lib().et_encode_batch_host_submit(enc.handle, _ptr(frames_host), offs.ctypes.data_as(_I32P), len(offs) - 1,
+                                             C.byref(q), _stream_ptr(stream), C.byref(dst.c), C.byref(ticket)),
+           enc.handle)
+    return HostCall(int(ticket.value), frames_host, dst)
+
+
+def et_encode_batch_host_collect(enc: Encoder, call: HostCall) -> Result:
+    r = et_result()
+    _check(lib().et_encode_batch_host_collect(enc.handle, C.c_ulonglong(call.ticket), C.byref(r)), enc.handle)
+    return _host_result(enc, r, call.dst)
 
 
 def et_kernel_launch_count() -> int:

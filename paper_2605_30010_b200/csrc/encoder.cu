@@ -98,7 +98,24 @@ struct et_encoder {
   AttnMaps attn_maps;                               // QKV as seen by the tcgen05 attention kernel
   bool attn_tc = false, scores_tc = false;
   float *lse = nullptr, *score_partial = nullptr, *scores = nullptr, *simbuf = nullptr;
-  float* frames_stage = nullptr;               // device staging for the *_host entry point (lazy)
+  // Pipelined host calls (et_encode_batch_host_submit / _collect): two calls may be in flight; each owns a slot with
+  // its own frame staging, result buffers and pinned words.  Slot 0's result buffers are the encoder's regular ones.
+  struct HostSlot {
+    float* frames_stage = nullptr;
+    float* tokens = nullptr;
+    int *token_pos = nullptr, *frame_offsets = nullptr, *src_lo = nullptr, *src_hi = nullptr, *vfo = nullptr;
+    unsigned char* dynamic = nullptr;
+    int *h_small = nullptr, *h_vid_off = nullptr;
+    cudaEvent_t ev_h2d = nullptr, ev_done = nullptr;
+    bool busy = false;                      // submitted and not collected yet
+    void* stream = nullptr;                 // the stream its work was enqueued on
+    et_params params{};
+    et_host_buffers dst{};
+    int V = 0, T = 0;
+    unsigned long long ticket = 0;
+  } slot[2];
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  unsigned long long next_ticket = 1;
 
   // frame lists, plans, traces
   FrameList fl[2]{};
@@ -282,9 +299,16 @@ SimPlanArgs sim_plan_args(et_encoder* e, const float* x, int n_cap, int lst, int
   return a;
 }
 
+et_status encode_finish(et_encoder* e, const et_params* p, int V, int T, int slot_idx, cudaStream_t s, et_result* out);
+
+// slot_idx selects the result buffers; with defer the call returns after enqueueing its work (the caller waits for
+// slot.ev_done and then calls encode_finish).
 et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off_host, int V, const et_params* p,
-                      cudaStream_t s, et_result* out) {
-  if (!e || !frames_dev || !vid_off_host || !out) return fail(e, ET_ERR_INVALID_ARG, "null argument");
+                      cudaStream_t s, et_result* out, int slot_idx = 0, bool defer = false) {
+  if (!e || !frames_dev || !vid_off_host || (!out && !defer)) return fail(e, ET_ERR_INVALID_ARG, "null argument");
+  et_encoder::HostSlot& sl = e->slot[slot_idx];
+  if (!defer && (e->slot[0].busy || e->slot[1].busy))
+    return fail(e, ET_ERR_INVALID_ARG, "a submitted call has not been collected yet");
   ET_TRY(validate_params(e, p) == ET_OK ? ET_OK : fail(e, ET_ERR_INVALID_ARG, "invalid et_params"));
   if (V < 1 || V > e->Vmax) return fail(e, ET_ERR_CAPACITY, "number of videos outside [1, max_videos]");
   if (vid_off_host[0] != 0) return fail(e, ET_ERR_INVALID_ARG, "video_offsets[0] must be 0");
@@ -313,8 +337,8 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
   const int rows_cap = T * L;
   const float* W = e->w_blob;
 
-  for (int v = 0; v <= V; ++v) e->h_vid_off[v] = vid_off_host[v] / e->tp;
-  ET_CUDA(e, cudaMemcpyAsync(e->orig_vid_off, e->h_vid_off, sizeof(int) * (V + 1), cudaMemcpyHostToDevice, s));
+  for (int v = 0; v <= V; ++v) sl.h_vid_off[v] = vid_off_host[v] / e->tp;
+  ET_CUDA(e, cudaMemcpyAsync(e->orig_vid_off, sl.h_vid_off, sizeof(int) * (V + 1), cudaMemcpyHostToDevice, s));
   ET_CUDA(e, cudaMemsetAsync(e->d_small, 0, sizeof(int) * 16, s));
   if (fp) {
     for (int i = 0; i < p->num_merge_layers; ++i) {
@@ -431,29 +455,47 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     }
     PROF(ET_CAT_SELECT, launch_select_video_tokens(sa, s));
   }
-  PROF(ET_CAT_GATHER, launch_gather_tokens(e->X[cur], e->keep, e->count, e->frame_offsets, e->d_small, T, L, D,
+  PROF(ET_CAT_GATHER, launch_gather_tokens(e->X[cur], e->keep, e->count, sl.frame_offsets, e->d_small, T, L, D,
                        c.post_layernorm ? W + e->off_post_g : nullptr, (c.post_layernorm && !qw) ? W + e->off_post_b : nullptr,
-                       c.ln_eps, e->tokens, e->token_pos, n_dev, s, e->raster2int));
-  ET_CUDA(e, cudaMemcpyAsync(e->h_small, e->d_small, sizeof(int) * 16, cudaMemcpyDeviceToHost, s));
+                       c.ln_eps, sl.tokens, sl.token_pos, n_dev, s, e->raster2int));
+  // per-frame results of this call: the frame list and flags are overwritten early in the next call
+  ET_CUDA(e, cudaMemcpyAsync(sl.src_lo, e->fl[lst].src_lo, sizeof(int) * T, cudaMemcpyDeviceToDevice, s));
+  ET_CUDA(e, cudaMemcpyAsync(sl.src_hi, e->fl[lst].src_hi, sizeof(int) * T, cudaMemcpyDeviceToDevice, s));
+  ET_CUDA(e, cudaMemcpyAsync(sl.dynamic, e->dynamic, T, cudaMemcpyDeviceToDevice, s));
+  ET_CUDA(e, cudaMemcpyAsync(sl.vfo, e->fl[lst].vid_off, sizeof(int) * (V + 1), cudaMemcpyDeviceToDevice, s));
+  ET_CUDA(e, cudaMemcpyAsync(sl.h_small, e->d_small, sizeof(int) * 16, cudaMemcpyDeviceToHost, s));
   ET_CUDA(e, cudaGetLastError());
+  if (defer) {
+    ET_CUDA(e, cudaEventRecord(sl.ev_done, s));
+    return ET_OK;
+  }
   ET_CUDA(e, cudaStreamSynchronize(s));
+  return encode_finish(e, p, V, T, slot_idx, s, out);
+}
 
-  const int status = e->h_small[10];
+// After the call's work has completed: status, sizes, result struct, profile counters, trace.
+et_status encode_finish(et_encoder* e, const et_params* p, int V, int T, int slot_idx, cudaStream_t s, et_result* out) {
+  et_encoder::HostSlot& sl = e->slot[slot_idx];
+  const et_config& c = e->cfg;
+  const int L = e->L, D = c.hidden, Mlp = c.mlp_dim;
+  const et_forced_plan* fp = p->forced_plan;
+  const bool qw = e->arch == 1;
+  const int status = sl.h_small[10];
   if (status == DS_WAIT_EXPIRED) return fail(e, ET_ERR_TIMEOUT, "a bounded device-side wait expired in a tensor-core kernel");
   if (status == DS_FORCED_MISMATCH) return fail(e, ET_ERR_INVALID_ARG, "forced plan does not fit the frame list");
   if (status != 0) return fail(e, ET_ERR_CUDA, "device status " + std::to_string(status));
-  const int N = e->h_small[0], n_tok = e->h_small[1];
+  const int N = sl.h_small[0], n_tok = sl.h_small[1];
   if (fp && fp->keep && fp->n_final != N) return fail(e, ET_ERR_INVALID_ARG, "forced plan: n_final does not match");
 
   et_result r{};
   r.n_videos = V; r.n_frames_in = T; r.n_frames_out = N; r.n_tokens = n_tok; r.hidden = D; r.tokens_per_frame = L;
-  r.tokens = e->tokens; r.video_frame_offsets = e->fl[lst].vid_off; r.frame_offsets = e->frame_offsets;
-  r.frame_src_lo = e->fl[lst].src_lo; r.frame_src_hi = e->fl[lst].src_hi; r.frame_dynamic = e->dynamic;
-  r.token_pos = e->token_pos; r.trace = nullptr;
+  r.tokens = sl.tokens; r.video_frame_offsets = sl.vfo; r.frame_offsets = sl.frame_offsets;
+  r.frame_src_lo = sl.src_lo; r.frame_src_hi = sl.src_hi; r.frame_dynamic = sl.dynamic;
+  r.token_pos = sl.token_pos; r.trace = nullptr;
   {
     int alive = T, m = 0;
     for (int layer = 0; layer < c.num_layers; ++layer) {
-      if (m < p->num_merge_layers && p->merge_layers[m] == layer) { alive = e->h_small[2 + m]; ++m; }
+      if (m < p->num_merge_layers && p->merge_layers[m] == layer) { alive = sl.h_small[2 + m]; ++m; }
       r.frames_per_block[layer] = alive;
     }
   }
@@ -471,7 +513,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     int n_in = T;
     for (int layer = 0, m = 0; layer < c.num_layers; ++layer) {
       if (m < p->num_merge_layers && p->merge_layers[m] == layer) {
-        const int n_out = e->h_small[2 + m];
+        const int n_out = sl.h_small[2 + m];
         wk[ET_CAT_SIMILARITY] += (double)n_in * dL * dD * 4.0;
         wk[ET_CAT_MERGE] += ((double)n_in + n_out) * dL * dD * 4.0;
         n_in = n_out; ++m;
@@ -494,7 +536,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     t.num_merge_layers = p->num_merge_layers;
     int n_in = T;
     for (int i = 0; i < p->num_merge_layers; ++i) {
-      t.n_in[i] = n_in; t.n_out[i] = e->h_small[2 + i];
+      t.n_in[i] = n_in; t.n_out[i] = sl.h_small[2 + i];
       float* hs = e->h_tr_f + (size_t)(2 * i) * e->Fmax;
       float* he = e->h_tr_f + (size_t)(2 * i + 1) * e->Fmax;
       unsigned char* hb = e->h_tr_b + (size_t)(2 * i) * e->Fmax;
@@ -655,6 +697,14 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
 #undef ET_A
   if ((st = halloc(e, &e->h_small, 16)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_vid_off, e->Vmax + 1)) != ET_OK) return bail(st);
+  {
+    et_encoder::HostSlot& s0 = e->slot[0];            // the slot of the synchronous calls: the regular result buffers
+    s0.tokens = e->tokens; s0.token_pos = e->token_pos; s0.frame_offsets = e->frame_offsets;
+    s0.h_small = e->h_small; s0.h_vid_off = e->h_vid_off;
+    if ((st = dalloc(e, &s0.src_lo, F)) != ET_OK || (st = dalloc(e, &s0.src_hi, F)) != ET_OK ||
+        (st = dalloc(e, &s0.dynamic, F)) != ET_OK || (st = dalloc(e, &s0.vfo, (size_t)e->Vmax + 1)) != ET_OK)
+      return bail(st);
+  }
   if ((st = halloc(e, &e->h_forced, 2 * ET_MAX_MERGE_LAYERS * F)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_keep_stage, rows)) != ET_OK) return bail(st);
   if ((st = halloc(e, &e->h_tr_f, 2 * ET_MAX_MERGE_LAYERS * F)) != ET_OK) return bail(st);
@@ -736,6 +786,11 @@ void et_destroy(et_encoder* e) {
   for (void* p : e->dev_allocs) cudaFree(p);
   for (void* p : e->host_allocs) cudaFreeHost(p);
   for (cudaEvent_t ev : e->prof_events) cudaEventDestroy(ev);
+  for (auto& sl : e->slot)
+    for (cudaEvent_t ev : {sl.ev_h2d, sl.ev_done})
+      if (ev) cudaEventDestroy(ev);
+  if (e->h2d_stream) cudaStreamDestroy(e->h2d_stream);
+  if (e->d2h_stream) cudaStreamDestroy(e->d2h_stream);
   delete e;
 }
 
@@ -751,18 +806,12 @@ et_status et_encode_video(et_encoder* enc, const float* frames_dev, int T, const
   return encode_impl(enc, frames_dev, offs, 1, params, (cudaStream_t)cuda_stream, out);
 }
 
-et_status et_encode_batch_host(et_encoder* e, const float* frames_host, const int* video_offsets_host, int V,
-                               const et_params* params, void* cuda_stream, const et_host_buffers* dst, et_result* out) {
-  if (!e || !frames_host || !video_offsets_host || !dst || !out) return fail(e, ET_ERR_INVALID_ARG, "null argument");
-  if (V < 1 || V > e->Vmax) return fail(e, ET_ERR_CAPACITY, "number of videos outside [1, max_videos]");
-  const int T = video_offsets_host[V];                     // input frames
-  if (T < 1 || T > e->Fmax * e->tp) return fail(e, ET_ERR_CAPACITY, "frames outside [1, max_frames_total]");
-  cudaStream_t s = (cudaStream_t)cuda_stream;
-  const size_t frame_floats = (size_t)3 * e->cfg.image_size * e->cfg.image_size;
-  if (!e->frames_stage) ET_TRY(dalloc(e, &e->frames_stage, (size_t)e->Fmax * e->tp * frame_floats));
-  ET_CUDA(e, cudaMemcpyAsync(e->frames_stage, frames_host, (size_t)T * frame_floats * sizeof(float), cudaMemcpyHostToDevice, s));
-  et_result r{};
-  ET_TRY(encode_impl(e, e->frames_stage, video_offsets_host, V, params, s, &r));
+}  // extern "C"
+
+namespace {
+
+// D2H of one call's results from its slot into the caller's host buffers, on stream s (not synchronised here)
+et_status copy_result_to_host(et_encoder* e, const et_result& r, int V, const et_host_buffers* dst, cudaStream_t s) {
   if ((size_t)r.n_tokens > dst->capacity_tokens || (size_t)r.n_frames_out > dst->capacity_frames)
     return fail(e, ET_ERR_CAPACITY, "host buffers too small for the result");
   const size_t N = r.n_frames_out, nt = r.n_tokens;
@@ -774,10 +823,112 @@ et_status et_encode_batch_host(et_encoder* e, const float* frames_host, const in
   if (dst->frame_dynamic) ET_CUDA(e, cudaMemcpyAsync(dst->frame_dynamic, r.frame_dynamic, N, cudaMemcpyDeviceToHost, s));
   if (dst->video_frame_offsets)
     ET_CUDA(e, cudaMemcpyAsync(dst->video_frame_offsets, r.video_frame_offsets, (V + 1) * sizeof(int), cudaMemcpyDeviceToHost, s));
+  return ET_OK;
+}
+
+et_status check_host_call(et_encoder* e, const float* frames_host, const int* video_offsets_host, int V, const et_host_buffers* dst) {
+  if (!e || !frames_host || !video_offsets_host || !dst) return fail(e, ET_ERR_INVALID_ARG, "null argument");
+  if (V < 1 || V > e->Vmax) return fail(e, ET_ERR_CAPACITY, "number of videos outside [1, max_videos]");
+  const int T = video_offsets_host[V];                     // input frames
+  if (T < 1 || T > e->Fmax * e->tp) return fail(e, ET_ERR_CAPACITY, "frames outside [1, max_frames_total]");
+  return ET_OK;
+}
+
+// Everything a slot needs beyond what create gave slot 0: frame staging, events, and for slot 1 result buffers of its own.
+et_status prepare_slot(et_encoder* e, int idx, bool events) {
+  et_encoder::HostSlot& sl = e->slot[idx];
+  const size_t F = e->Fmax, rows = F * (size_t)e->L, D = e->cfg.hidden;
+  const size_t frame_floats = (size_t)3 * e->cfg.image_size * e->cfg.image_size;
+  if (!sl.frames_stage) ET_TRY(dalloc(e, &sl.frames_stage, F * e->tp * frame_floats));
+  if (!sl.tokens) {
+    ET_TRY(dalloc(e, &sl.tokens, rows * D)); ET_TRY(dalloc(e, &sl.token_pos, rows)); ET_TRY(dalloc(e, &sl.frame_offsets, F + 1));
+    ET_TRY(dalloc(e, &sl.src_lo, F)); ET_TRY(dalloc(e, &sl.src_hi, F)); ET_TRY(dalloc(e, &sl.dynamic, F));
+    ET_TRY(dalloc(e, &sl.vfo, (size_t)e->Vmax + 1));
+    ET_TRY(halloc(e, &sl.h_small, 16)); ET_TRY(halloc(e, &sl.h_vid_off, (size_t)e->Vmax + 1));
+  }
+  if (events && !sl.ev_done) {
+    ET_CUDA(e, cudaEventCreateWithFlags(&sl.ev_h2d, cudaEventDisableTiming));
+    ET_CUDA(e, cudaEventCreateWithFlags(&sl.ev_done, cudaEventDisableTiming));
+  }
+  return ET_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+et_status et_encode_batch_host(et_encoder* e, const float* frames_host, const int* video_offsets_host, int V,
+                               const et_params* params, void* cuda_stream, const et_host_buffers* dst, et_result* out) {
+  if (!out) return fail(e, ET_ERR_INVALID_ARG, "null argument");
+  ET_TRY(check_host_call(e, frames_host, video_offsets_host, V, dst));
+  const int T = video_offsets_host[V];
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const size_t frame_floats = (size_t)3 * e->cfg.image_size * e->cfg.image_size;
+  ET_CUDA(e, cudaSetDevice(e->device));
+  ET_TRY(prepare_slot(e, 0, false));
+  ET_CUDA(e, cudaMemcpyAsync(e->slot[0].frames_stage, frames_host, (size_t)T * frame_floats * sizeof(float), cudaMemcpyHostToDevice, s));
+  et_result r{};
+  ET_TRY(encode_impl(e, e->slot[0].frames_stage, video_offsets_host, V, params, s, &r));
+  ET_TRY(copy_result_to_host(e, r, V, dst, s));
   ET_CUDA(e, cudaStreamSynchronize(s));
   *out = r;
   return ET_OK;
 }
+
+et_status et_encode_batch_host_submit(et_encoder* e, const float* frames_host, const int* video_offsets_host, int V,
+                                      const et_params* params, void* cuda_stream, const et_host_buffers* dst,
+                                      unsigned long long* ticket) {
+  if (!ticket || !params) return fail(e, ET_ERR_INVALID_ARG, "null argument");
+  ET_TRY(check_host_call(e, frames_host, video_offsets_host, V, dst));
+  if (params->forced_plan || params->want_trace) return fail(e, ET_ERR_INVALID_ARG, "forced plans and traces need the synchronous calls");
+  if (e->prof_on) return fail(e, ET_ERR_INVALID_ARG, "per-category profiling needs the synchronous calls");
+  const int idx = (int)(e->next_ticket & 1ull);
+  et_encoder::HostSlot& sl = e->slot[idx];
+  if (sl.busy) return fail(e, ET_ERR_CAPACITY, "two calls are in flight already: collect the older one first");
+  if (e->slot[idx ^ 1].busy && e->slot[idx ^ 1].stream != cuda_stream)
+    return fail(e, ET_ERR_INVALID_ARG, "calls in flight together must use one stream: they share the encoder's work buffers");
+  const int T = video_offsets_host[V];
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const size_t frame_floats = (size_t)3 * e->cfg.image_size * e->cfg.image_size;
+  ET_CUDA(e, cudaSetDevice(e->device));
+  ET_TRY(prepare_slot(e, idx, true));
+  if (!e->h2d_stream) {
+    ET_CUDA(e, cudaStreamCreateWithFlags(&e->h2d_stream, cudaStreamNonBlocking));
+    ET_CUDA(e, cudaStreamCreateWithFlags(&e->d2h_stream, cudaStreamNonBlocking));
+  }
+  // Upload on the copy stream, compute behind the upload.  The slot's previous call has been collected, so nothing
+  // reads its staging area or result buffers any more.
+  ET_CUDA(e, cudaMemcpyAsync(sl.frames_stage, frames_host, (size_t)T * frame_floats * sizeof(float), cudaMemcpyHostToDevice, e->h2d_stream));
+  ET_CUDA(e, cudaEventRecord(sl.ev_h2d, e->h2d_stream));
+  ET_CUDA(e, cudaStreamWaitEvent(s, sl.ev_h2d, 0));
+  ET_TRY(encode_impl(e, sl.frames_stage, video_offsets_host, V, params, s, nullptr, idx, true));
+  sl.params = *params; sl.dst = *dst; sl.V = V; sl.T = T / e->tp; sl.stream = cuda_stream; sl.busy = true;
+  sl.ticket = e->next_ticket++;
+  *ticket = sl.ticket;
+  return ET_OK;
+}
+
+et_status et_encode_batch_host_collect(et_encoder* e, unsigned long long ticket, et_result* out) {
+  if (!e || !out) return fail(e, ET_ERR_INVALID_ARG, "null argument");
+  const int idx = (int)(ticket & 1ull);
+  et_encoder::HostSlot& sl = e->slot[idx];
+  if (!sl.busy || sl.ticket != ticket) return fail(e, ET_ERR_INVALID_ARG, "no such call in flight");
+  const et_encoder::HostSlot& other = e->slot[idx ^ 1];
+  if (other.busy && other.ticket < ticket) return fail(e, ET_ERR_INVALID_ARG, "collect the older call first");
+  ET_CUDA(e, cudaSetDevice(e->device));
+  sl.busy = false;                                 // whatever happens below, the slot is free again
+  ET_CUDA(e, cudaEventSynchronize(sl.ev_done));
+  et_result r{};
+  ET_TRY(encode_finish(e, &sl.params, sl.V, sl.T, idx, nullptr, &r));
+  ET_TRY(copy_result_to_host(e, r, sl.V, &sl.dst, e->d2h_stream));
+  ET_CUDA(e, cudaStreamSynchronize(e->d2h_stream));
+  *out = r;
+  return ET_OK;
+}
+
+}  // extern "C"
+
+extern "C" {
 
 const char* et_status_string(et_status s) {
   switch (s) {

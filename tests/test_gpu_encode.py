@@ -175,6 +175,79 @@ def test_host_entry_point_matches_device_entry_point(B):
     enc.close()
 
 
+def test_pipelined_host_calls_match_synchronous_calls(B):
+    """Two host calls in flight (submit, submit, collect, submit, ...) give bit for bit what the synchronous host call
+    gives, on videos of different lengths and content, in both architectures' slot rotation; misuse is refused."""
+    import torch
+    from synthetic.videos import make_video
+    wl = workload("tiny")
+    s = wl.shape
+    blob = make_weights(s, wl.weight_seed)
+    enc = B.Encoder(s, blob, B.ET_F32, 8)
+    vids = [torch.from_numpy(make_video(n, s.image_size, s.patch_size, p, seed)).pin_memory()
+            for n, p, seed in ((8, 0.3, 0), (5, 0.6, 1), (7, 0.1, 2), (8, 0.9, 3), (3, 0.3, 4))]
+    want = []
+    for v in vids:
+        dst = B.HostBuffers(8 * 64, 8, s.hidden)
+        r = B.et_encode_batch_host(enc, v, [0, v.shape[0]], wl.params, dst)
+        want.append((r.n_tokens, r.n_frames_out, r.tokens.clone(), r.token_pos.clone(), r.frame_offsets.clone(),
+                     r.frame_src_lo.clone(), r.frame_src_hi.clone(), r.frame_dynamic.clone()))
+    assert len({w[0] for w in want}) > 1                      # the calls really differ
+    bufs = [B.HostBuffers(8 * 64, 8, s.hidden) for _ in range(2)]
+    stream = torch.cuda.Stream()
+    got, calls = [], []
+    for i, v in enumerate(vids):
+        calls.append(B.et_encode_batch_host_submit(enc, v, [0, v.shape[0]], wl.params, bufs[i % 2], stream))
+        if len(calls) == 2:
+            r = B.et_encode_batch_host_collect(enc, calls.pop(0))
+            got.append((r.n_tokens, r.n_frames_out, r.tokens.clone(), r.token_pos.clone(), r.frame_offsets.clone(),
+                        r.frame_src_lo.clone(), r.frame_src_hi.clone(), r.frame_dynamic.clone()))
+    r = B.et_encode_batch_host_collect(enc, calls.pop(0))
+    got.append((r.n_tokens, r.n_frames_out, r.tokens.clone(), r.token_pos.clone(), r.frame_offsets.clone(),
+                r.frame_src_lo.clone(), r.frame_src_hi.clone(), r.frame_dynamic.clone()))
+    assert len(got) == len(want)
+    for g, w in zip(got, want):
+        assert g[0] == w[0] and g[1] == w[1]
+        for a, b in zip(g[2:], w[2:]):
+            assert torch.equal(a, b)
+
+    # misuse: a third call in flight, collecting out of order, an unknown ticket, a synchronous call in between,
+    # another stream, a trace request
+    c1 = B.et_encode_batch_host_submit(enc, vids[0], [0, 8], wl.params, bufs[0], stream)
+    with pytest.raises(B.EarlyTomError) as ei:
+        B.et_encode_batch_host_submit(enc, vids[1], [0, 5], wl.params, bufs[1], torch.cuda.Stream())
+    assert ei.value.status == 1
+    c2 = B.et_encode_batch_host_submit(enc, vids[1], [0, 5], wl.params, bufs[1], stream)
+    with pytest.raises(B.EarlyTomError) as ei:
+        B.et_encode_batch_host_submit(enc, vids[2], [0, 7], wl.params, B.HostBuffers(8 * 64, 8, s.hidden), stream)
+    assert ei.value.status == 3
+    with pytest.raises(B.EarlyTomError) as ei:
+        B.et_encode_batch_host_collect(enc, c2)
+    assert ei.value.status == 1
+    with pytest.raises(B.EarlyTomError) as ei:
+        enc.encode_video(to_cuda(vids[0].numpy()), wl.params)
+    assert ei.value.status == 1
+    r1 = B.et_encode_batch_host_collect(enc, c1)
+    assert r1.n_tokens == want[0][0] and torch.equal(r1.tokens, want[0][2])
+    with pytest.raises(B.EarlyTomError) as ei:
+        B.et_encode_batch_host_collect(enc, c1)
+    assert ei.value.status == 1
+    r2 = B.et_encode_batch_host_collect(enc, c2)
+    assert r2.n_tokens == want[1][0] and torch.equal(r2.tokens, want[1][2])
+    import ctypes as C
+    q, _keep = B.make_params(wl.params, None, True)           # a trace request, through the raw entry point
+    offs8 = np.array([0, 8], dtype=np.int32)
+    ticket = C.c_ulonglong(0)
+    st = B.lib().et_encode_batch_host_submit(enc.handle, C.c_void_p(vids[0].data_ptr()),
+                                             offs8.ctypes.data_as(C.POINTER(C.c_int32)), 1, C.byref(q), None,
+                                             C.byref(bufs[0].c), C.byref(ticket))
+    assert st == 1
+    # the encoder still serves synchronous calls afterwards
+    dev = enc.encode_video(to_cuda(vids[0].numpy()), wl.params)
+    assert dev.n_tokens == want[0][0] and torch.equal(dev.tokens.cpu(), want[0][2])
+    enc.close()
+
+
 def test_argument_errors(B):
     wl = workload("tiny")
     frames, offs = make_batch(wl)
