@@ -131,11 +131,14 @@ void launch_attention_bf16(const bf16* qkv, bf16* out, float* lse, int n_cap, in
                            const int* n_frames_dev, cudaStream_t s);
 bool attention_bf16_supported(int L, int heads, int dh);
 // tcgen05 attention (attention_tcgen05.cu): head dims 64, 72 and 80.  The maps describe qkv [rows][3*D] bf16.
-struct AttnMaps { TmaDesc main, tail; };
+// Q boxes (128 rows), K / V boxes (one key tile), and the attention output as [frames][L][D] (stores clipped per frame)
+struct AttnMaps { TmaDesc main, tail, kv_main, kv_tail, out; };
 bool attention_tc_supported(int dh);
-bool make_attention_maps(AttnMaps* out, const bf16* qkv, long long rows, int heads, int dh);
-// window_rows > 0: a query attends only to the keys of its run of window_rows consecutive rows of the frame
-cudaError_t launch_attention_tc(const AttnMaps& maps, bf16* out, float* lse, int n_cap, int L, int heads, int dh,
+// attn_out (with the tokens per frame L) may be NULL for users that only read Q / K / V through the maps
+bool make_attention_maps(AttnMaps* out, const bf16* qkv, long long rows, int heads, int dh, bf16* attn_out = nullptr, int L = 0);
+// The output goes where maps.out points.  window_rows > 0: a query attends only to the keys of its run of
+// window_rows consecutive rows of the frame
+cudaError_t launch_attention_tc(const AttnMaps& maps, float* lse, int n_cap, int L, int heads, int dh,
                                 const int* n_frames_dev, int* status_dev, cudaStream_t s, int window_rows = 0);
 bool attention_scores_tc_supported(int dh);
 // partial[f][h][j] = sum_q exp(s(q,j) - lse[f][h][q]);  score[f][j] = sum_h partial / (heads*L)

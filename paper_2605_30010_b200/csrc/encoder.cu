@@ -393,7 +393,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
     const int* a_n = windowed ? e->n_windows : n_dev;
     PROF(ET_CAT_ATTENTION, {
       // the tensor-core kernel sweeps whole frames and masks the keys outside a query's window
-      if (e->attn_tc) ET_CUDA(e, launch_attention_tc(e->attn_maps, (bf16*)e->O, e->lse, T, L, H, dh, n_dev, e->d_small + 10, s, windowed ? e->Lw : 0));
+      if (e->attn_tc) ET_CUDA(e, launch_attention_tc(e->attn_maps, e->lse, T, L, H, dh, n_dev, e->d_small + 10, s, windowed ? e->Lw : 0));
       else if (e->bf) launch_attention_bf16((const bf16*)e->QKV, (bf16*)e->O, e->lse, a_cap, a_L, H, dh, a_n, s);
       else launch_attention_f32((const float*)e->QKV, (float*)e->O, e->lse, a_cap, a_L, H, dh, a_n, s);
     });
@@ -770,7 +770,7 @@ et_status et_encoder_create(const et_config* config, const et_weights* weights, 
       if (cudaMemcpy(e->bgu_pad, hb.data(), hb.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) return bail(ET_ERR_CUDA);
     }
     if (attention_tc_supported(e->dh)) {
-      if (!make_attention_maps(&e->attn_maps, (const bf16*)e->QKV, (long long)rows, config->heads, e->dh))
+      if (!make_attention_maps(&e->attn_maps, (const bf16*)e->QKV, (long long)rows, config->heads, e->dh, (bf16*)e->O, e->L))
         return bail(fail(e, ET_ERR_CUDA, "tensor map of the attention operands"));
       e->attn_tc = true;
       e->scores_tc = attention_scores_tc_supported(e->dh);
@@ -1089,8 +1089,8 @@ et_status et_attention(const void* qkv_dev, void* out_dev, float* lse_dev, int n
     if (head_dim % 8 != 0) return ET_ERR_SHAPE;
     if (attention_tc_supported(head_dim)) {
       AttnMaps maps;
-      if (!make_attention_maps(&maps, (const bf16*)qkv_dev, (long long)n * L, heads, head_dim)) return ET_ERR_CUDA;
-      ET_CUDA0(launch_attention_tc(maps, (bf16*)out_dev, lse_dev, n, L, heads, head_dim, nullptr, nullptr, s));
+      if (!make_attention_maps(&maps, (const bf16*)qkv_dev, (long long)n * L, heads, head_dim, (bf16*)out_dev, L)) return ET_ERR_CUDA;
+      ET_CUDA0(launch_attention_tc(maps, lse_dev, n, L, heads, head_dim, nullptr, nullptr, s));
       return ET_OK;
     }
     launch_attention_bf16((const bf16*)qkv_dev, (bf16*)out_dev, lse_dev, n, L, heads, head_dim, nullptr, s);
@@ -1114,8 +1114,8 @@ et_status et_attention_windowed(const void* qkv_dev, void* out_dev, float* lse_s
     if (head_dim % 8 != 0) return ET_ERR_SHAPE;
     if (attention_tc_supported(head_dim)) {
       AttnMaps maps;
-      if (!make_attention_maps(&maps, (const bf16*)qkv_dev, (long long)n * L, heads, head_dim)) return ET_ERR_CUDA;
-      ET_CUDA0(launch_attention_tc(maps, (bf16*)out_dev, lse_scratch_dev, n, L, heads, head_dim, nullptr, nullptr, s, window_rows));
+      if (!make_attention_maps(&maps, (const bf16*)qkv_dev, (long long)n * L, heads, head_dim, (bf16*)out_dev, L)) return ET_ERR_CUDA;
+      ET_CUDA0(launch_attention_tc(maps, lse_scratch_dev, n, L, heads, head_dim, nullptr, nullptr, s, window_rows));
       return ET_OK;
     }
     launch_attention_bf16((const bf16*)qkv_dev, (bf16*)out_dev, lse_scratch_dev, items, window_rows, heads, head_dim, nullptr, s);
