@@ -2,6 +2,7 @@
 // weighted merge with frame compaction (Eq. 3).  All HBM-bound or latency-bound; no tensor cores.
 #include "common.cuh"
 #include "rowops.cuh"
+#include "tcgen05.cuh"
 
 namespace et {
 
@@ -327,12 +328,12 @@ void launch_merge_plan(const PlanArgs& a, int n_cap, cudaStream_t s) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Similarities and plan in ONE launch (the encoder's path).  Jobs are the (run of 8 pairs, position) items of
-// token_cos_kernel.  The mean over positions is accumulated without any scratch array and without any order:
+// Similarities and plan in ONE launch (the encoder's path).  A block job is a run of 8 pairs over a strip of
+// positions; the cosine of a (pair, position) is computed as in token_cos_kernel.  The mean over positions is accumulated without any scratch array and without any order:
 // every cosine is scaled by 2^32, rounded to an integer and added to the pair's 64-bit accumulator with an atomic
 // add.  Integer addition is exact and commutative, so the result does not depend on the order of arrival (bit-
 // reproducible), and the rounding step (2^-32 per position) is far below the fp32 rounding of the cosine itself.
-// Nobody waits for anybody: a block that has finished all its jobs takes one ticket; the block that takes the last
+// No block waits for another: a block that has finished all its jobs takes one ticket; the block that takes the last
 // ticket turns the accumulators into similarities (resetting them for the next launch) and runs the plan
 // (Eq. 1-2, Eq. 3 weights, next list).  Pairs that straddle two videos are not computed.
 // ---------------------------------------------------------------------------------------------
@@ -341,13 +342,33 @@ constexpr double SIM_FIXED_ONE = 4294967296.0;     // 2^32
 // work on the same few pairs at the same time, and thousands of atomic adds to one address queue up in one L2 slice.
 constexpr int SIM_SLOTS = 16;
 
+// The frames are streamed through shared memory by a producer warp: a block job is a strip of S consecutive positions
+// over a run of frames; the strip of one frame is contiguous in memory (S rows of D floats) and comes in with ONE bulk
+// copy (cp.async.bulk, completion on an mbarrier) into a ring of frame slots.  Consumer warp w owns position w of the
+// strip: it reads its row of the current and of the previous frame from shared memory, reduces as cos_run does (same
+// arithmetic, same order), and releases the previous frame's slot, which the producer refills at once.  The bytes in
+// flight per SM are a whole slot, whatever the registers hold, and issuing the copies costs the consumers nothing
+// (with plain loads, a row per warp under way, the kernel reached 0.55 of the copy bandwidth; a bulk copy per row
+// issued by the consuming warp itself cost that warp 600 cycles per row).
+constexpr int SIM_MAX_STRIP = 16;                  // consumer warps = positions per strip
+constexpr int SIM_MAX_SLOTS = 8;
+constexpr int SIM_SMEM_BUDGET = 222 * 1024;
+
+__device__ __forceinline__ void bulk_load_rows(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
 template <int NV>
-__global__ void __launch_bounds__(128) similarity_plan_kernel(SimPlanArgs a) {
-  extern __shared__ int sh_plan[];      // used only by the block that runs the plan
+__global__ void __launch_bounds__((SIM_MAX_STRIP + 1) * 32, 1)
+similarity_plan_kernel(SimPlanArgs a, int plan_bytes, int strip, int slots) {
+  extern __shared__ __align__(128) unsigned char sh_raw[];
+  int* const sh_plan = reinterpret_cast<int*>(sh_raw);      // used only by the block that runs the plan
   __shared__ unsigned sh_last;
+  __shared__ int sh_abort;
   const int n = min(*a.n_frames_dev, a.n_cap);
   const int n_pairs = n - 1;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int stage = min(a.n_cap, PLAN_STAGE_FRAMES);
   if (n_pairs <= 0) {                   // single frame: nothing to compare, the plan still sets roles and counts
     if (blockIdx.x == 0) {
@@ -357,32 +378,113 @@ __global__ void __launch_bounds__(128) similarity_plan_kernel(SimPlanArgs a) {
     }
     return;
   }
+  const int n_strips = (a.L + strip - 1) / strip;
   const int n_runs = (n_pairs + COS_RUN - 1) / COS_RUN;
-  const int n_jobs = n_runs * a.L;
-  if (blockIdx.x * wpb >= n_jobs) return;               // blocks without a job take no ticket
-  const int warps_total = gridDim.x * wpb;
-  const int* vo = a.vid_off;
-  int v = 0;                            // video of the current frame; jobs of a warp come in ascending frame order
-  for (int job = blockIdx.x * wpb + warp; job < n_jobs; job += warps_total) {
-    const int l = job % a.L, run = job / a.L;
-    const int t0 = run * COS_RUN, t1 = min(t0 + COS_RUN, n_pairs);
-    ET_CHECK(t0 >= 0 && t1 <= a.n_cap - 1 && t0 < vo[a.n_videos], continue);
-    unsigned cross = 0;                 // bit q: frames t0+q and t0+q+1 belong to different videos
-    for (int t = t0; t < t1; ++t) {
-      while (vo[v + 1] <= t) ++v;
-      if (t + 1 == vo[v + 1]) cross |= 1u << (t - t0);
+  const int n_jobs = n_runs * n_strips;
+  if ((int)blockIdx.x >= n_jobs) return;                // blocks without a job take no ticket
+  const uint32_t row_bytes = (uint32_t)a.D * 4u;
+  const size_t slot_bytes = (size_t)strip * row_bytes;
+  const uint32_t bar_full = tc::smem_u32(sh_raw + plan_bytes), bar_empty = bar_full + 8u * SIM_MAX_SLOTS;
+  unsigned char* const ring = sh_raw + plan_bytes + 1024;
+  if (threadIdx.x == 0) {
+    sh_abort = 0;
+    for (int i = 0; i < slots; ++i) { tc::mbar_init(bar_full + 8u * i, 1); tc::mbar_init(bar_empty + 8u * i, (uint32_t)strip); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  bool ok = true;
+  if (warp == strip) {
+    // ---- producer: the frames t0 .. t1 of every job of this block, in order, one copy each
+    int slot = 0, uses = 0;
+    uint32_t phase = 1;                 // parity of the release that precedes a slot's use (none before its first)
+    for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+      const int run = job / n_strips, l0 = (job % n_strips) * strip;
+      const int t0 = run * COS_RUN, t1 = min(t0 + COS_RUN, n_pairs);
+      const uint32_t bytes = (uint32_t)min(strip, a.L - l0) * row_bytes;
+      ET_CHECK(t0 >= 0 && t1 <= a.n_cap - 1 && l0 < a.L, ok = false);
+      if (!ok) break;
+      for (int t = t0; t <= t1; ++t, ++uses) {
+        if (uses >= slots && !tc::mbar_wait_warp(bar_empty + 8u * slot, phase, &sh_abort)) { ok = false; break; }
+        if (lane == 0) {
+          tc::mbar_arrive_expect_tx(bar_full + 8u * slot, bytes);
+          bulk_load_rows(tc::smem_u32(ring + (size_t)slot * slot_bytes), a.x + ((size_t)t * a.L + l0) * a.D, bytes, bar_full + 8u * slot);
+        }
+        if (++slot == slots) { slot = 0; phase ^= 1u; }
+      }
     }
-    auto is_cross = [cross, t0](int t) { return ((cross >> (t - t0)) & 1u) != 0; };
-    unsigned long long* acc = a.acc + (size_t)(l % SIM_SLOTS) * a.n_cap;
-    cos_run<NV>(a.x, l, t0, t1, a.L, a.D, lane, is_cross, [=](int t, float c) {
-      // c * 2^32 is exact in fp32 (a power-of-two scaling), so the only rounding is the one to an integer
-      if (lane == 0) atomicAdd(acc + t, (unsigned long long)__float2ll_rn(c * 4294967296.0f));
-    });
+  } else if (warp < strip) {
+    // ---- consumers
+    const int nvec = a.D >> 2;
+    const int* vo = a.vid_off;
+    int v = 0;                          // video of the current frame; the jobs of a block come in ascending frame order
+    int slot = 0;                       // ring position and phase of the next frame
+    uint32_t phase = 0;
+    for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+      const int run = job / n_strips, l = (job % n_strips) * strip + warp;
+      const int t0 = run * COS_RUN, t1 = min(t0 + COS_RUN, n_pairs);
+      const bool mine = l < a.L;        // the last strip of a frame may be short: its spare warps only pass the slots on
+      unsigned cross = 0;               // bit q: frames t0+q and t0+q+1 belong to different videos
+      for (int t = t0; t < t1; ++t) {
+        while (vo[v + 1] <= t) ++v;
+        if (t + 1 == vo[v + 1]) cross |= 1u << (t - t0);
+      }
+      float4 prev[NV];                  // the previous frame's row stays in registers: a slot is free once it has been read
+      float np = 0.f;
+      float my_dot = 0.f, my_np = 1.f, my_nc = 1.f;      // lane q keeps the sums of pair t0 + q until the run is done
+      for (int r = 0; r <= t1 - t0; ++r) {
+        if (!tc::mbar_wait_warp(bar_full + 8u * slot, phase, &sh_abort)) { ok = false; break; }
+        float4 cur[NV];
+        if (mine) {
+          const float4* row = reinterpret_cast<const float4*>(ring + (size_t)slot * slot_bytes + (size_t)warp * row_bytes);
+#pragma unroll
+          for (int j = 0; j < NV; ++j) {
+            const int i = lane + 32 * j;
+            cur[j] = (i < nvec) ? row[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
+        __syncwarp();                   // every lane has taken its part of the row
+        if (lane == 0) tc::mbar_arrive(bar_empty + 8u * slot);
+        if (++slot == slots) { slot = 0; phase ^= 1u; }
+        if (mine) {
+          float dot = 0.f, nc = 0.f;
+          if (r == 0) {
+#pragma unroll
+            for (int j = 0; j < NV; ++j)
+              nc += (cur[j].x * cur[j].x + cur[j].y * cur[j].y) + (cur[j].z * cur[j].z + cur[j].w * cur[j].w);
+            nc = warp_sum(nc);
+          } else {
+#pragma unroll
+            for (int j = 0; j < NV; ++j) {
+              const float4 c = cur[j];
+              dot += (prev[j].x * c.x + prev[j].y * c.y) + (prev[j].z * c.z + prev[j].w * c.w);
+              nc += (c.x * c.x + c.y * c.y) + (c.z * c.z + c.w * c.w);
+            }
+            dot = warp_sum(dot);
+            nc = warp_sum(nc);
+            if (lane == r - 1) { my_dot = dot; my_np = np; my_nc = nc; }
+          }
+          np = nc;
+#pragma unroll
+          for (int j = 0; j < NV; ++j) prev[j] = cur[j];
+        }
+      }
+      if (ok && mine && lane < t1 - t0 && !((cross >> lane) & 1u)) {
+        // c * 2^32 is exact in fp32 (a power-of-two scaling), so the only rounding is the one to an integer
+        const float c = my_dot / fmaxf(sqrtf(my_np) * sqrtf(my_nc), 1e-8f);
+        atomicAdd(a.acc + (size_t)(l % SIM_SLOTS) * a.n_cap + (t0 + lane), (unsigned long long)__float2ll_rn(c * 4294967296.0f));
+      }
+    }
+  }
+  if (!ok) {                            // a wait ran out: report it, and give the copies in flight time to land
+    if (lane == 0) atomicExch(a.plan.status, (int)DS_WAIT_EXPIRED);
+    const unsigned long long t_begin = tc::global_ns();
+    while (tc::global_ns() - t_begin < 200000ull) __nanosleep(1000);
   }
   if (lane == 0) __threadfence();       // this warp's additions before the block's ticket
   __syncthreads();
   if (threadIdx.x == 0) {
-    const unsigned blocks_with_jobs = (unsigned)min((long long)gridDim.x, ((long long)n_jobs + wpb - 1) / wpb);
+    const unsigned blocks_with_jobs = (unsigned)min((int)gridDim.x, n_jobs);
     sh_last = atomicAdd(a.done, 1u) == blocks_with_jobs - 1u ? 1u : 0u;
   }
   __syncthreads();
@@ -413,11 +515,31 @@ int similarity_plan_words(int n_cap) { return SIM_SLOTS * n_cap + 1; }
 
 void launch_similarity_plan(const SimPlanArgs& a, cudaStream_t s) {
   const int runs = max(1, cdiv(max(a.n_cap - 1, 1), COS_RUN));
-  const int blocks = max(1, min(cdiv((long long)runs * a.L, 4), 148 * 16));
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
   const int need = cdiv(a.D / 4, 32);
-  const size_t smem = plan_smem_bytes(a.n_videos, a.n_cap);
+  const int plan_bytes = (int)((plan_smem_bytes(a.n_videos, a.n_cap) + 127) & ~(size_t)127);
+  const int row_bytes = a.D * 4;
+  // the strip as wide as three slots (the frame being read, two on their way) allow; then as many slots as fit
+  const int room = SIM_SMEM_BUDGET - plan_bytes - 1024;
+  const int strip = max(1, min(min(SIM_MAX_STRIP, a.L), room / (3 * row_bytes)));
+  const int slots = max(2, min(SIM_MAX_SLOTS, room / (strip * row_bytes)));
+  const size_t smem = (size_t)plan_bytes + 1024 + (size_t)slots * strip * row_bytes;
+  const int blocks = (int)max(1ll, min((long long)runs * cdiv(a.L, strip), (long long)sms));   // one block per SM
   ET_COUNT_LAUNCH();
-#define ET_SP(NV) similarity_plan_kernel<NV><<<blocks, 128, smem, s>>>(a)
+#define ET_SP(NV)                                                                                                     \
+  do {                                                                                                                \
+    static bool configured = false;                                                                                   \
+    if (!configured) {                                                                                                \
+      cudaFuncSetAttribute(similarity_plan_kernel<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, SIM_SMEM_BUDGET); \
+      configured = true;                                                                                              \
+    }                                                                                                                 \
+    similarity_plan_kernel<NV><<<blocks, (strip + 1) * 32, smem, s>>>(a, plan_bytes, strip, slots);                   \
+  } while (0)
   if (need <= 1) ET_SP(1);
   else if (need <= 2) ET_SP(2);
   else if (need <= 4) ET_SP(4);
