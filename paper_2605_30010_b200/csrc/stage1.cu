@@ -152,14 +152,15 @@ static inline size_t plan_smem_bytes(int n_videos, int n_cap) {
 // Per-frame flag byte while the plan is being made
 enum : unsigned char { PF_START = 1, PF_MERGE = 2, PF_LAST = 4, PF_FIRST = 8 };
 
-// The plan of one merge layer, executed by ONE warp (lane = 0..31).  Shared memory: sh_count [n_videos + 1] ints
-// followed by the staging area for `stage_frames` frames (similarity, EMA, source range, flag byte).
-//   phase A, a lane per video, frames in order: the EMA recurrence of Eq. 1 with its restarts, and the pairing of
-//            Eq. 2 inside each segment, are chains in which a step depends on the decision before it.  They only
-//            touch the staged arrays (a chain of reads from global memory would cost a memory latency per frame);
-//   phase B, a lane per frame: everything that depends on one frame and its neighbour -- the output index (a prefix
-//            sum of "this frame opens an output frame" by ballot / popc), the Eq. 3 weights, the source ranges and
-//            roles of the next list, the trace.
+// The plan of one merge layer, executed by ALL threads of a block (it synchronises them).  Shared memory: sh_count
+// [n_videos + 1] ints followed by the staging area for `stage_frames` frames (similarity, EMA, source range, flag byte).
+//   phase A, a thread per video (the first videos on lane 0 of each warp, so that their chains do not diverge),
+//            frames in order: the EMA recurrence of Eq. 1 with its restarts, and the pairing of Eq. 2 inside each
+//            segment, are chains in which a step depends on the decision before it.  They only touch the staged
+//            arrays (a chain of reads from global memory would cost a memory latency per frame);
+//   phase B, a warp per video and a lane per frame: everything that depends on one frame and its neighbour -- the
+//            output index (the video's offset plus a prefix sum of "this frame opens an output frame" by ballot /
+//            popc), the Eq. 3 weights, the source ranges and roles of the next list, the trace.
 // Lists longer than the staging area work on the global arrays (the trace arrays double as working storage).
 // Similarities are read past the L1 (other SMs may have written them during the same kernel).
 // Copies the list's similarities and source ranges into the staging area (any number of threads; the caller
@@ -177,11 +178,12 @@ __device__ __forceinline__ void merge_plan_stage(const PlanArgs& a, int tid, int
   }
 }
 
-__device__ void merge_plan_body(const PlanArgs& a, int lane, int* sh_count, int stage_frames) {
+__device__ void merge_plan_body(const PlanArgs& a, int tid, int nthr, int* sh_count, int stage_frames) {
+  const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
   const int V = a.n_videos;
   const int n = *a.cur.n;
   const bool forced = a.forced_seg_start != nullptr;
-  if (forced && lane == 0 && a.forced_n_in != n) atomicExch(a.status, (int)DS_FORCED_MISMATCH);
+  if (forced && tid == 0 && a.forced_n_in != n) atomicExch(a.status, (int)DS_FORCED_MISMATCH);
   const bool use_forced = forced && a.forced_n_in == n;
   const bool staged = n <= stage_frames;
   float* const st_sim = reinterpret_cast<float*>(sh_count + V + 1);
@@ -195,8 +197,8 @@ __device__ void merge_plan_body(const PlanArgs& a, int lane, int* sh_count, int 
   auto lo_at = [&](int t) -> int { return staged ? st_lo[t] : a.cur.src_lo[t]; };
   auto hi_at = [&](int t) -> int { return staged ? st_hi[t] : a.cur.src_hi[t]; };
 
-  // ---- phase A: per video, in frame order
-  for (int v = lane; v < V; v += 32) {
+  // ---- phase A: per video, in frame order (video v on lane v / nwarps of warp v % nwarps)
+  for (int v = warp + nwarps * lane; v < V; v += nwarps * 32) {
     const int g0 = a.cur.vid_off[v], g1 = a.cur.vid_off[v + 1];
     double prev = 0.0;
     bool have_prev = false;
@@ -246,19 +248,21 @@ __device__ void merge_plan_body(const PlanArgs& a, int lane, int* sh_count, int 
     }
     sh_count[v] = out;
   }
-  __syncwarp();
-  if (lane == 0) {                                     // offsets of the next list
+  __syncthreads();
+  if (tid == 0) {                                      // offsets of the next list
     int acc = 0;
     for (int v = 0; v < V; ++v) { const int c = sh_count[v]; sh_count[v] = acc; acc += c; }
     sh_count[V] = acc;
   }
-  __syncwarp();
+  __syncthreads();
 
-  // ---- phase B: per frame
-  int carry = 0;                                       // output frames before this chunk of 32 input frames
-  for (int base = 0; base < n; base += 32) {
+  // ---- phase B: per frame, a warp per video
+  for (int v = warp; v < V; v += nwarps) {
+  const int g0 = a.cur.vid_off[v], g1 = a.cur.vid_off[v + 1];
+  int carry = sh_count[v];                             // output frames before this chunk of 32 input frames
+  for (int base = g0; base < g1; base += 32) {
     const int t = base + lane;
-    const bool live = t < n;
+    const bool live = t < g1;
     const unsigned char f = live ? flag[t] : 0;
     const unsigned char fp = (live && t > 0) ? flag[t - 1] : 0;
     const unsigned char fn = (live && t + 1 < n) ? flag[t + 1] : 0;
@@ -302,14 +306,15 @@ __device__ void merge_plan_body(const PlanArgs& a, int lane, int* sh_count, int 
     if (staged) a.trace.ema[t] = ema[t];
     a.trace.merge_next[t] = mrg ? 1 : 0;
   }
-  __syncwarp();                                        // every neighbour's flag has been read
-  for (int t = lane; t < n; t += 32) a.trace.seg_start[t] = (flag[t] & PF_START) ? 1 : 0;
+  }
+  __syncthreads();                                     // every neighbour's flag has been read
+  for (int t = tid; t < n; t += nthr) a.trace.seg_start[t] = (flag[t] & PF_START) ? 1 : 0;
   if (!a.allow_merge) {
-    if (lane == 0 && a.n_hist_slot) *a.n_hist_slot = n;
+    if (tid == 0 && a.n_hist_slot) *a.n_hist_slot = n;
     return;
   }
-  for (int v = lane; v <= V; v += 32) a.nxt.vid_off[v] = sh_count[v];
-  if (lane == 0) {
+  for (int v = tid; v <= V; v += nthr) a.nxt.vid_off[v] = sh_count[v];
+  if (tid == 0) {
     *a.nxt.n = sh_count[V];
     if (a.n_hist_slot) *a.n_hist_slot = sh_count[V];
   }
@@ -319,7 +324,7 @@ __global__ void merge_plan_kernel(PlanArgs a, int stage_frames) {
   extern __shared__ int sh_plan_count[];
   merge_plan_stage(a, threadIdx.x, blockDim.x, sh_plan_count, stage_frames);
   __syncthreads();
-  if (threadIdx.x < 32) merge_plan_body(a, threadIdx.x, sh_plan_count, stage_frames);
+  merge_plan_body(a, threadIdx.x, blockDim.x, sh_plan_count, stage_frames);
 }
 
 void launch_merge_plan(const PlanArgs& a, int n_cap, cudaStream_t s) {
@@ -374,7 +379,7 @@ similarity_plan_kernel(SimPlanArgs a, int plan_bytes, int strip, int slots) {
     if (blockIdx.x == 0) {
       merge_plan_stage(a.plan, threadIdx.x, blockDim.x, sh_plan, stage);
       __syncthreads();
-      if (warp == 0) merge_plan_body(a.plan, lane, sh_plan, stage);
+      merge_plan_body(a.plan, threadIdx.x, blockDim.x, sh_plan, stage);
     }
     return;
   }
@@ -508,7 +513,7 @@ similarity_plan_kernel(SimPlanArgs a, int plan_bytes, int strip, int slots) {
   __syncthreads();
   merge_plan_stage(a.plan, threadIdx.x, blockDim.x, sh_plan, stage);
   __syncthreads();
-  if (warp == 0) merge_plan_body(a.plan, lane, sh_plan, stage);
+  merge_plan_body(a.plan, threadIdx.x, blockDim.x, sh_plan, stage);
 }
 
 int similarity_plan_words(int n_cap) { return SIM_SLOTS * n_cap + 1; }
