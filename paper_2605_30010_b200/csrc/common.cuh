@@ -154,8 +154,9 @@ cudaError_t launch_attention_scores_tc(const AttnMaps& maps, const float* lse, f
 // attention_causal_tcgen05.cu: causal grouped-query attention, head dim 128, over packed rows
 // [heads*128 | kv_heads*128 | kv_heads*128] of n_seq sequences of L positions each.
 bool attention_causal_supported(int head_dim);
-bool make_causal_attention_map(TmaDesc* out, const bf16* qkv, long long rows, int heads, int kv_heads);
-cudaError_t launch_attention_causal(const TmaDesc& map, bf16* out, int n_seq, int L, int heads, int kv_heads,
+struct CausalMaps { TmaDesc q, kv; };     // the packed Q | K | V rows in boxes of 128 rows (Q) and of one key tile (K, V)
+bool make_causal_attention_map(CausalMaps* out, const bf16* qkv, long long rows, int heads, int kv_heads);
+cudaError_t launch_attention_causal(const CausalMaps& map, bf16* out, int n_seq, int L, int heads, int kv_heads,
                                     int* status_dev, cudaStream_t s);
 
 // ---- llm_ops.cu: row-wise and elementwise steps of the language model --------------------------

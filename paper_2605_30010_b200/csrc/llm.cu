@@ -359,7 +359,7 @@ et_status et_llm_prefill(et_llm* m, const int* prefix_ids_host, int n_prefix, co
   }
 
   // ---- decoder layers
-  TmaDesc attn_map;
+  CausalMaps attn_map;
   if (!make_causal_attention_map(&attn_map, m->QKV, n, c.heads, c.kv_heads)) return lfail(m, ET_ERR_CUDA, "tensor map of the attention operands");
   int layer_index = 0;
   for (const LlmLayer& l : m->layers) {
@@ -467,7 +467,7 @@ et_status et_attention_causal(const void* qkv_dev, void* out_dev, int n_seq, int
   if (!qkv_dev || !out_dev) return ET_ERR_INVALID_ARG;
   if (n_seq < 1 || L < 1 || heads < 1 || kv_heads < 1 || heads % kv_heads != 0 || !attention_causal_supported(head_dim)) return ET_ERR_SHAPE;
   if ((long long)n_seq * L > (1ll << 30)) return ET_ERR_CAPACITY;
-  TmaDesc map;
+  CausalMaps map;
   if (!make_causal_attention_map(&map, (const bf16*)qkv_dev, (long long)n_seq * L, heads, kv_heads)) return ET_ERR_CUDA;
   return launch_attention_causal(map, (bf16*)out_dev, n_seq, L, heads, kv_heads, status_dev, (cudaStream_t)cuda_stream) == cudaSuccess
              ? ET_OK : ET_ERR_CUDA;
