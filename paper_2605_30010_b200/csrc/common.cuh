@@ -84,7 +84,8 @@ enum Epilogue : int { EPI_STORE = 0, EPI_GELU = 1, EPI_RESIDUAL = 2, EPI_TABLE =
 // frames fp32 [T][3][H][W] -> patches [T*L][k_pad] (zero padded beyond 3*p*p), fp32 or bf16.
 // tp input frames make one encoder frame (T counts encoder frames); int2raster: optional internal token order.
 void launch_im2col(const float* frames, void* patches, int T, int image, int patch, int k_pad, bool out_bf16,
-                   const int* n_frames_dev, cudaStream_t s, int tp = 1, const int* int2raster = nullptr);
+                   const int* n_frames_dev, cudaStream_t s, int tp = 1, const int* int2raster = nullptr,
+                   const int* raster2int = nullptr);   // both token-order tables or neither
 // 2-D rotary positions in place on the Q and K parts of packed rows [rows][3*heads*dh]; table [L][dh/2] (cos, sin)
 void launch_rope_pairs(void* qkv, const float2* table, int rows_cap, int L, int heads, int dh, bool is_bf16,
                        const int* n_frames_dev, cudaStream_t s);

@@ -53,9 +53,63 @@ __global__ void im2col_kernel(const float* __restrict__ frames, T* __restrict__ 
   }
 }
 
+// The same result with the work laid out along the image: a warp takes one pixel row of one channel of one input
+// frame, reads it as consecutive pixel pairs (coalesced) and scatters the pairs to the patch rows they belong to (runs
+// of `patch` elements); further warps write the zero pad of 32 tokens each.  Needs even patch, image and k_pad and
+// 8-byte aligned frames; `raster2int` is the inverse of the order im2col_kernel takes (NULL: raster order).
+template <typename T>
+__global__ void im2col_rows_kernel(const float* __restrict__ frames, T* __restrict__ patches, int T_frames, int image,
+                                   int patch, int grid, int k_pad, int tp, const int* __restrict__ raster2int,
+                                   const int* __restrict__ n_frames_dev) {
+  const int n_frames = n_frames_dev ? min(*n_frames_dev, T_frames) : T_frames;      // encoder frames
+  const int L = grid * grid, crop = grid * patch, K = 3 * tp * patch * patch;
+  const int lane = threadIdx.x & 31;
+  const long long row_jobs = (long long)n_frames * tp * 3 * crop;
+  const long long pad_jobs = K < k_pad ? ((long long)n_frames * L + 31) / 32 : 0;
+  const long long warps = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long job = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); job < row_jobs + pad_jobs; job += warps) {
+    if (job >= row_jobs) {
+      const long long tok = (job - row_jobs) * 32 + lane;
+      if (tok < (long long)n_frames * L)
+        for (int c = K; c < k_pad; ++c) patches[tok * k_pad + c] = to_out<T>(0.f);
+      continue;
+    }
+    const int y = (int)(job % crop);
+    const long long fc = job / crop;                    // (input frame, channel)
+    const int c = (int)(fc % 3);
+    const long long f_in = fc / 3;
+    const int t = (int)(f_in % tp);
+    const long long f = f_in / tp;
+    const int gy = y / patch, dy = y - gy * patch;
+    const float2* src = reinterpret_cast<const float2*>(frames + ((f_in * 3 + c) * image + y) * image);
+    T* const dst_frame = patches + f * L * (long long)k_pad + ((c * tp + t) * patch + dy) * patch;
+    for (int x = 2 * lane; x < crop; x += 64) {
+      const float2 v = __ldg(src + (x >> 1));
+      const int gx = x / patch, dx = x - gx * patch;
+      int l = gy * grid + gx;
+      if (raster2int) l = raster2int[l];
+      store_pair(dst_frame + (long long)l * k_pad + dx, v.x, v.y);
+    }
+  }
+}
+
 void launch_im2col(const float* frames, void* patches, int T, int image, int patch, int k_pad, bool out_bf16,
-                   const int* n_frames_dev, cudaStream_t s, int tp, const int* int2raster) {
+                   const int* n_frames_dev, cudaStream_t s, int tp, const int* int2raster, const int* raster2int) {
   const int grid = image / patch;
+  if ((patch & 1) == 0 && (image & 1) == 0 && (k_pad & 1) == 0 && (reinterpret_cast<size_t>(frames) & 7) == 0 &&
+      (int2raster == nullptr) == (raster2int == nullptr)) {
+    const long long jobs = (long long)T * tp * 3 * grid * patch + ((long long)T * grid * grid + 31) / 32;
+    const int threads = 256;
+    const long long want = (jobs + 7) / 8;
+    const int blocks = (int)(want < 148LL * 32 ? want : 148LL * 32);
+    if (blocks == 0) return;
+    ET_COUNT_LAUNCH();
+    if (out_bf16)
+      im2col_rows_kernel<bf16><<<blocks, threads, 0, s>>>(frames, (bf16*)patches, T, image, patch, grid, k_pad, tp, raster2int, n_frames_dev);
+    else
+      im2col_rows_kernel<float><<<blocks, threads, 0, s>>>(frames, (float*)patches, T, image, patch, grid, k_pad, tp, raster2int, n_frames_dev);
+    return;
+  }
   const long long total = (long long)T * grid * grid * (3 * tp * patch + 1);
   const int threads = 256;
   long long want = (total + threads - 1) / threads;

@@ -357,7 +357,7 @@ et_status encode_impl(et_encoder* e, const float* frames_dev, const int* vid_off
 
   // patch embedding: im2col + dense layer with the position table added in the epilogue
   const bool qw = e->arch == 1;           // Qwen2.5-VL-style blocks
-  PROF(ET_CAT_IM2COL, launch_im2col(frames_dev, e->Pm, T, c.image_size, c.patch_size, e->Kp, e->bf, nullptr, s, e->tp, e->int2raster));
+  PROF(ET_CAT_IM2COL, launch_im2col(frames_dev, e->Pm, T, c.image_size, c.patch_size, e->Kp, e->bf, nullptr, s, e->tp, e->int2raster, e->raster2int));
   PROF(ET_CAT_GEMM, ET_TRY(dense(e, e->Pm, e->d_Pm, W + e->off_patch_w, e->d_patch_w, e->c_X[cur], qw ? e->zeros : W + e->off_patch_b, e->X[cur], rows_cap, D,
                e->bf ? e->Kp : e->P, EPI_TABLE, qw ? e->zeros : W + e->off_pos, qw ? 1 : L, nullptr, s)));
   if (e->ws > 0) launch_scale_count(e->fl[0].n, e->wpf, e->n_windows, s);
